@@ -1,0 +1,501 @@
+"""Pins for the CPU oracle: closed forms, brute force, invariants and the paper's printed numbers.
+
+None of these tests touches the CUDA path; they establish that ``oracle/`` computes what the
+paper defines before anything is compared against it.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2601_17818_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16(x):
+    return W.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+# =============================================================================== O1: K-norm (Eq. 4)
+def test_knorm_constant_closed_form():
+    # all entries c  ->  |c| * sqrt(H*d);  c = 1, H = 32, d = 128  ->  exactly 64
+    K = bf16(np.ones((2, 32, 5, 128)))
+    s = oracle.knorm(K, 0, 5)
+    assert np.array_equal(s, np.full((2, 5), 64.0))
+    K = bf16(np.full((1, 8, 3, 64), -0.5))
+    assert np.array_equal(oracle.knorm(K, 0, 3), np.full((1, 3), 0.5 * math.sqrt(8 * 64)))
+
+
+def test_knorm_one_hot_and_zero():
+    K = np.zeros((1, 4, 6, 16), dtype=np.float32)
+    K[0, 2, 3, 7] = -3.0
+    K[0, 1, 4, 0] = 0.375
+    s = oracle.knorm(bf16(K), 0, 6)[0]
+    assert s[3] == 3.0 and s[4] == 0.375
+    assert np.all(s[[0, 1, 2, 5]] == 0.0)
+
+
+def test_knorm_equals_frobenius_norm_of_flattened_row():
+    rng = np.random.default_rng(1)
+    Kf = W.bf16_bits_to_f32(bf16(rng.standard_normal((3, 5, 11, 24))))
+    s = oracle.knorm(bf16(Kf), 0, 11)
+    flat = np.transpose(Kf.astype(np.float64), (0, 2, 1, 3)).reshape(3, 11, -1)
+    ref = np.linalg.norm(flat, axis=-1)                 # textbook L2 norm of the concatenated heads
+    np.testing.assert_allclose(s, ref, rtol=1e-14)
+
+
+def test_knorm_span_and_invariances():
+    rng = np.random.default_rng(2)
+    Kf = W.bf16_bits_to_f32(bf16(rng.standard_normal((2, 6, 20, 16))))
+    full = oracle.knorm(bf16(Kf), 0, 20)
+    part = oracle.knorm(bf16(Kf), 7, 9)                 # only the visual span [7, 16) is scored
+    assert np.array_equal(part, full[:, 7:16])
+    ragged = oracle.knorm(bf16(Kf), 3, np.array([4, 10], dtype=np.int32))
+    assert np.array_equal(ragged[0, :4], full[0, 3:7]) and np.array_equal(ragged[1], full[1, 3:13])
+    # permuting heads or elements changes only the summation order
+    perm_h = oracle.knorm(bf16(Kf[:, ::-1]), 0, 20)
+    perm_e = oracle.knorm(bf16(Kf[..., ::-1]), 0, 20)
+    np.testing.assert_allclose(perm_h, full, rtol=1e-14)
+    np.testing.assert_allclose(perm_e, full, rtol=1e-14)
+    # scaling by a power of two is exact
+    assert np.array_equal(oracle.knorm(bf16(Kf * 8.0), 0, 20), full * 8.0)
+
+
+def test_knorm_is_rotation_invariant():
+    # rotating (e_2t, e_2t+1) pairs (RoPE) leaves the norm unchanged; done in float64 before
+    # rounding is impossible in bf16, so check the identity on exactly representable rotations (90 degrees)
+    rng = np.random.default_rng(3)
+    Kf = W.bf16_bits_to_f32(bf16(rng.standard_normal((1, 2, 4, 8))))
+    rot = np.empty_like(Kf)
+    rot[..., 0::2] = -Kf[..., 1::2]
+    rot[..., 1::2] = Kf[..., 0::2]
+    np.testing.assert_allclose(oracle.knorm(bf16(rot), 0, 4), oracle.knorm(bf16(Kf), 0, 4), rtol=1e-14)
+
+
+# =============================================================================== O2: plain top-k
+def _is_valid_topk(score, kept, k, largest=False):
+    """Definition: |S| = k and every kept (score, index) pair precedes every dropped pair."""
+    n = len(score)
+    kept = set(int(i) for i in kept)
+    if len(kept) != min(k, n):
+        return False
+    key = [((-s if largest else s), i) for i, s in enumerate(score)]
+    drop = [key[i] for i in range(n) if i not in kept]
+    keep = [key[i] for i in kept]
+    return not keep or not drop or max(keep) < min(drop)
+
+
+@pytest.mark.parametrize("kind", ["lognormal", "ties", "equal", "signed"])
+def test_select_plain_brute_force(kind):
+    for n in (1, 2, 5, 9, 12):
+        score = W.make_scores(5, 1, n, kind)[0].astype(np.float64)
+        for k in range(0, n + 3):
+            for largest in (False, True):
+                got = oracle.select_plain(score, k, largest)
+                assert list(got) == sorted(got), "ascending output"
+                assert _is_valid_topk(score, got, k, largest)
+                # uniqueness of the valid set: enumerate every subset of that size
+                kk = min(k, n)
+                valid = [c for c in itertools.combinations(range(n), kk) if _is_valid_topk(score, c, k, largest)]
+                assert valid == [tuple(got)]
+
+
+def test_select_plain_monotone_inputs():
+    n, k = 17, 6
+    inc = np.arange(n, dtype=np.float64)
+    assert list(oracle.select_plain(inc, k)) == list(range(k))
+    assert list(oracle.select_plain(-inc, k)) == list(range(n - k, n))
+    assert list(oracle.select_plain(np.ones(n), k)) == list(range(k))           # ties -> lowest index
+    assert list(oracle.select_plain(inc, 0)) == []
+    assert list(oracle.select_plain(inc, n)) == list(range(n))
+    assert list(oracle.select_plain(inc, n + 5)) == list(range(n))              # budget >= n keeps everything
+    s = W.make_scores(3, 1, 40, "signed")[0].astype(np.float64)
+    assert np.array_equal(oracle.select_plain(s, 11, largest=True), oracle.select_plain(-s, 11))
+
+
+def test_select_smaller_norm_is_kept():
+    # Stage III keeps the tokens with the SMALLEST K-norm
+    s = np.array([5.0, 1.0, 4.0, 0.5, 3.0])
+    assert list(oracle.select_plain(s, 2)) == [1, 3]
+
+
+def test_select_nan_sorts_last():
+    s = np.array([2.0, np.nan, 1.0, np.inf, 0.0])
+    assert list(oracle.select_plain(s, 3)) == [0, 2, 4]
+    assert list(oracle.select_plain(s, 4)) == [0, 2, 3, 4]
+
+
+# =============================================================================== O4: quota (Eq. 5)
+def _read_quota_examples():
+    out = []
+    with open(os.path.join(GOLDEN, "quota_examples.txt")) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            b, sizes, q = [p.strip() for p in line.split(";")]
+            out.append((int(b), [int(x) for x in sizes.split()], [int(x) for x in q.split()]))
+    return out
+
+
+def test_quota_hand_examples():
+    for budget, sizes, quotas in _read_quota_examples():
+        n = sum(sizes)
+        # cluster c occupies a contiguous run; its label is the run's first token
+        label = np.concatenate([np.full(s, sum(sizes[:c]), dtype=np.int32) for c, s in enumerate(sizes)])
+        score = np.arange(n, dtype=np.float64)[::-1].copy()
+        keep, nc, quota = oracle.select_quota(score, label, budget)
+        assert nc == len(sizes)
+        got_q = [int(quota[sum(sizes[:c])]) for c in range(len(sizes))]
+        assert got_q == quotas
+        assert len(keep) == sum(quotas) and len(keep) + nc <= budget
+        # decreasing scores -> each cluster keeps its LAST q_c members
+        start = 0
+        expect = []
+        for s, q in zip(sizes, quotas):
+            expect += list(range(start + s - q, start + s))
+            start += s
+        assert list(keep) == expect
+
+
+def test_quota_single_cluster_equals_plain():
+    s = W.make_scores(11, 1, 50, "lognormal")[0].astype(np.float64)
+    label = np.full(50, 17, dtype=np.int32)
+    keep, nc, _ = oracle.select_quota(s, label, 20)
+    assert nc == 1
+    assert np.array_equal(keep, oracle.select_plain(s, 19))        # q = (50 * 19) div 50 = 19
+
+
+@pytest.mark.parametrize("kind", ["lognormal", "ties"])
+def test_quota_properties_random(kind):
+    n, ncl = 97, 7
+    s = W.make_scores(4, 1, n, kind)[0].astype(np.float64)
+    label = W.make_labels(4, 1, n, ncl)[0]
+    for budget in (ncl, ncl + 1, 30, 60, n):
+        keep, nc, quota = oracle.select_quota(s, label, budget)
+        assert nc == len(set(label.tolist()))
+        total = 0
+        for c in set(label.tolist()):
+            members = np.flatnonzero(label == c)
+            q = (len(members) * (budget - nc)) // n                 # Eq. 5 in integers
+            assert quota[c] == q
+            kept_c = [i for i in keep if label[i] == c]
+            assert len(kept_c) == q
+            local = [int(np.flatnonzero(members == i)[0]) for i in kept_c]
+            assert _is_valid_topk(s[members], local, q)             # definitional check inside the cluster
+            total += q
+        assert len(keep) == total <= budget - nc
+        assert list(keep) == sorted(keep)
+    assert oracle.select_quota(s, label, ncl - 1)[0] is None        # budget below the cluster count
+
+
+# =============================================================================== O3: VIC (Alg. 2)
+def _unit_rows(n, D, seed):
+    rng = np.random.default_rng(seed)
+    return bf16(rng.standard_normal((n, D)))
+
+
+def test_similarity_basic_properties():
+    f = _unit_rows(40, 64, 0)
+    d2, sim = oracle.feature_distance(f, 0)
+    np.testing.assert_allclose(np.diag(sim), 1.0, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(sim, sim.T, rtol=0, atol=1e-15)
+    assert np.all(np.abs(sim) <= 1 + 1e-15)
+    np.testing.assert_allclose(d2, np.maximum(0, 2 - 2 * sim), atol=1e-15)
+    # cosine distance is the Euclidean distance between the L2-normalised rows (numpy, independent route)
+    x = W.bf16_bits_to_f32(f).astype(np.float64)
+    xn = x / np.linalg.norm(x, axis=1, keepdims=True)
+    ref = ((xn[:, None, :] - xn[None, :, :]) ** 2).sum(-1)
+    np.testing.assert_allclose(d2, ref, atol=1e-13)
+    # euclid metric: plain squared distance; "sim" is then the raw Gram matrix
+    d2e, g = oracle.feature_distance(f, 1)
+    np.testing.assert_allclose(d2e, ((x[:, None, :] - x[None, :, :]) ** 2).sum(-1), rtol=1e-12, atol=1e-10)
+    np.testing.assert_allclose(g, x @ x.T, rtol=1e-12, atol=1e-12)
+    # a row block equals the same rows of the full matrix
+    d2r, simr = oracle.feature_distance(f, 0, rows=(7, 19))
+    assert np.array_equal(d2r, d2[7:19]) and np.array_equal(simr, sim[7:19])
+
+
+def test_similarity_hand_values():
+    # f0 = (1,0), f1 = (1,1), f2 = (0,2), f3 = (-1,0):  cos(0,1) = 1/sqrt2, cos(0,2) = 0, cos(0,3) = -1
+    f = bf16([[1, 0], [1, 1], [0, 2], [-1, 0]])
+    d2, sim = oracle.feature_distance(f, 0)
+    r = 1 / math.sqrt(2)
+    np.testing.assert_allclose(sim[0], [1, r, 0, -1], atol=1e-15)
+    np.testing.assert_allclose(d2[0], [0, 2 - 2 * r, 2, 4], atol=1e-15)
+    np.testing.assert_allclose(sim[1, 2], r, atol=1e-15)
+    # Eq. 2 by hand for token 0 with d_c = 0.5
+    rho = oracle.vic_density(d2, 0.5)
+    expect0 = math.exp(-(2 - 2 * r) / 0.25) + math.exp(-2 / 0.25) + math.exp(-4 / 0.25)
+    assert abs(rho[0] - expect0) < 1e-15
+    # zero-norm feature: similarity 0 against everything, d2 = 2
+    d2z, simz = oracle.feature_distance(bf16([[0, 0], [1, 0]]), 0)
+    assert simz[0, 1] == 0 and d2z[0, 1] == 2
+
+
+def test_density_closed_forms():
+    n, dc = 16, 0.7
+    eye = bf16(np.eye(n) * 3.0)                         # orthogonal rows: s = 0, d^2 = 2
+    d2, _ = oracle.feature_distance(eye, 0)
+    assert np.all(d2[~np.eye(n, dtype=bool)] == 2.0)
+    rho = oracle.vic_density(d2, dc)
+    np.testing.assert_allclose(rho, (n - 1) * math.exp(-2 / dc ** 2), rtol=1e-14)
+    same = bf16(np.tile(np.array([[1.0, -2.0, 0.5]]), (n, 1)))   # n identical tokens: every term is exp(0)
+    d2s, _ = oracle.feature_distance(same, 0)
+    np.testing.assert_allclose(d2s, 0, atol=1e-15)
+    np.testing.assert_allclose(oracle.vic_density(d2s, dc), n - 1, rtol=1e-14)
+
+
+def test_identical_tokens_single_cluster():
+    n = 9
+    f = bf16(np.tile(np.array([[1.0, 2.0, 3.0, 4.0]]), (n, 1)))
+    r = oracle.vic(f, None, 0, 0.5, -1.0, 1)
+    assert r["is_center"].tolist() == [1] + [0] * (n - 1)   # equal densities: the lowest index is densest
+    assert np.all(r["label"] == 0)
+    assert r["parent"].tolist() == [-1] + [0] * (n - 1)     # ties in distance -> lowest index
+    assert math.isinf(r["delta2"][0]) and np.all(r["delta2"][1:] < 1e-15)
+
+
+def test_exact_duplicates_share_a_cluster():
+    w = W.workload("tiny")
+    f = W.make_features(w)[0].copy()
+    p = W.make_positions(w)[0]
+    f[31] = f[30]                                        # neighbours on the 24-grid, inside tau
+    f[101] = f[100]
+    r = oracle.vic(f, p, 0, w.d_c, w.tau, w.n_centers)
+    assert r["sim"][30, 31] == pytest.approx(1.0, abs=1e-15) and r["d2"][30, 31] < 1e-15
+    assert r["label"][30] == r["label"][31] and r["label"][100] == r["label"][101]
+
+
+def test_two_separated_groups():
+    rng = np.random.default_rng(5)
+    a = np.array([1.0, 0, 0, 0]) + 0.02 * rng.standard_normal((6, 4))
+    b = np.array([0, 0, 1.0, 0]) + 0.02 * rng.standard_normal((8, 4))
+    f = bf16(np.concatenate([a, b]))
+    r = oracle.vic(f, None, 0, 0.5, -1.0, 2)
+    la, lb = set(r["label"][:6].tolist()), set(r["label"][6:].tolist())
+    assert len(la) == 1 and len(lb) == 1 and la != lb
+    assert list(la)[0] < 6 <= list(lb)[0]                # each label is a token of its own group
+
+
+def _density_peaks_bruteforce(x, dc, n_centers):
+    """Independent restatement (pure Python) of density-peaks clustering with a Gaussian kernel."""
+    n = len(x)
+    xn = [v / np.linalg.norm(v) for v in x]
+    d = [[float(np.linalg.norm(xn[i] - xn[j])) for j in range(n)] for i in range(n)]
+    rho = [sum(math.exp(-(d[i][j] / dc) ** 2) for j in range(n) if j != i) for i in range(n)]
+    parent, delta = [], []
+    for i in range(n):
+        cand = [(d[i][j], j) for j in range(n) if j != i and (rho[j] > rho[i] or (rho[j] == rho[i] and j < i))]
+        if cand:
+            dd, j = min(cand)
+            parent.append(j), delta.append(dd)
+        else:
+            parent.append(-1), delta.append(math.inf)
+    gamma = [rho[i] * delta[i] if parent[i] >= 0 else math.inf for i in range(n)]
+    order = sorted(range(n), key=lambda i: (-gamma[i], -rho[i], i))
+    centres = set(order[:n_centers])
+    label = [-1] * n
+    for i in sorted(range(n), key=lambda i: (-rho[i], i)):
+        if i in centres:
+            label[i] = i
+        elif parent[i] >= 0:
+            label[i] = label[parent[i]]
+        else:
+            label[i] = min((d[i][c], c) for c in centres)[1]
+    return rho, delta, parent, sorted(centres), label
+
+
+@pytest.mark.parametrize("seed,n,nc", [(0, 24, 3), (1, 48, 5), (2, 64, 4)])
+def test_vic_without_spatial_mask_is_density_peaks(seed, n, nc):
+    rng = np.random.default_rng(seed)
+    centres = rng.standard_normal((nc, 12))
+    x = centres[rng.integers(0, nc, n)] + 0.3 * rng.standard_normal((n, 12))
+    fb = bf16(x)
+    xf = W.bf16_bits_to_f32(fb).astype(np.float64)
+    rho, delta, parent, cs, label = _density_peaks_bruteforce(xf, 0.5, nc)
+    pos = rng.random((n, 2)).astype(np.float32)
+    for kwargs in (dict(pos=None, tau=-1.0), dict(pos=pos, tau=1e9)):        # tau = infinity: mask is vacuous
+        r = oracle.vic(fb, kwargs["pos"], 0, 0.5, kwargs["tau"], nc)
+        np.testing.assert_allclose(r["rho"], rho, rtol=1e-12)
+        assert r["parent"].tolist() == parent
+        fin = np.isfinite(r["delta2"])
+        np.testing.assert_allclose(np.sqrt(r["delta2"][fin]), np.array(delta)[fin], atol=1e-7)
+        assert np.flatnonzero(r["is_center"]).tolist() == cs
+        assert r["label"].tolist() == label
+
+
+def test_spatial_mask_hand_example():
+    # unit vectors at angles 0, 0.1, 0.2, 0.9 rad: chord distance ~ angle, so with d_c = 0.5 the
+    # densities fall in the order 1 > 2 > 0 > 3 (token 1 sits in the middle of the tight triple)
+    ang = np.array([0.0, 0.1, 0.2, 0.9])
+    f = bf16(np.stack([np.cos(ang), np.sin(ang)], 1))
+    d2, _ = oracle.feature_distance(f, 0)
+    rho = oracle.vic_density(d2, 0.5)
+    assert sorted(range(4), key=lambda i: -rho[i]) == [1, 2, 0, 3]
+    # no mask: everybody points at the nearest denser token in feature space
+    delta2, parent, _ = oracle.vic_parents(d2, None, rho, -1.0)
+    assert parent.tolist() == [1, -1, 1, 2] and math.isinf(delta2[1])
+    assert delta2[3] == d2[3, 2] and delta2[0] == d2[0, 1]
+    # tokens laid out on a line at x = 0, 0.1, 0.9, 1.0
+    pos = np.array([[0.0, 0.0], [0.1, 0.0], [0.9, 0.0], [1.0, 0.0]], dtype=np.float32)
+    # tau = 0.15: 3 sees only 2; 0 sees only 1; 2 sees only 3 (less dense) and 1 only 0 (less dense)
+    delta2, parent, _ = oracle.vic_parents(d2, pos, rho, 0.15)
+    assert parent.tolist() == [1, -1, -1, 2] and math.isinf(delta2[2])
+    # tau = 0.05: nobody sees anybody
+    delta2, parent, _ = oracle.vic_parents(d2, pos, rho, 0.05)
+    assert parent.tolist() == [-1] * 4 and np.all(np.isinf(delta2))
+    # the mask redirects token 0: its nearest denser token (1) is far away in the image, token 2 is close
+    pos = np.array([[0.0, 0.0], [1.0, 0.0], [0.1, 0.0], [0.5, 0.5]], dtype=np.float32)
+    delta2, parent, _ = oracle.vic_parents(d2, pos, rho, 0.5)
+    assert parent[0] == 2 and delta2[0] == d2[0, 2] and delta2[0] > d2[0, 1]
+    # a pair exactly tau apart is admitted ("<= tau"), just below it is not
+    pos = np.array([[0.0, 0.0], [0.5, 0.0], [0.0, 0.75], [0.75, 0.75]], dtype=np.float32)
+    assert oracle.vic_parents(d2, pos, rho, 0.5)[1][0] == 1
+    assert oracle.vic_parents(d2, pos, rho, 0.4999)[1][0] == -1
+
+
+def test_all_orphans_fall_back_to_nearest_centre():
+    w = W.workload("tiny")
+    f = W.make_features(w)[0][:60]
+    p = W.make_positions(w)[0][:60]
+    r = oracle.vic(f, p, 0, w.d_c, 0.0, 5)               # tau = 0, distinct positions: no admissible neighbour
+    assert np.all(r["parent"] == -1) and np.all(np.isinf(r["delta2"]))
+    cs = np.flatnonzero(r["is_center"])
+    assert cs.tolist() == sorted(np.argsort(-r["rho"], kind="stable")[:5].tolist())   # orphans rank by density
+    for i in range(60):
+        if i in cs:
+            assert r["label"][i] == i
+        else:
+            assert r["label"][i] == cs[np.argmin(r["d2"][i, cs])]
+
+
+@pytest.mark.parametrize("name", ["tiny", "c0"])
+def test_vic_invariants(name):
+    w = W.workload(name)
+    f = W.make_features(w)[0]
+    p = W.make_positions(w)[0]
+    r = oracle.vic(f, p, 0, w.d_c, w.tau, w.n_centers)
+    n = f.shape[0]
+    rho, parent, label = r["rho"], r["parent"], r["label"]
+    cs = set(np.flatnonzero(r["is_center"]).tolist())
+    assert len(cs) == w.n_centers == r["n_clusters"]
+    assert set(label.tolist()) == cs                     # every label is a centre, every centre is used
+    for i in range(n):
+        j = parent[i]
+        if j >= 0:
+            assert rho[j] > rho[i] or (rho[j] == rho[i] and j < i)          # chains climb in density: no cycles
+            assert np.hypot(*(p[i].astype(np.float64) - p[j].astype(np.float64))) <= w.tau
+            assert r["delta2"][i] == r["d2"][i, j]
+        if i in cs:
+            assert label[i] == i
+        elif j >= 0:
+            assert label[i] == label[j]
+    # permuting feature dimensions or scaling by a power of two changes nothing discrete
+    perm = np.random.default_rng(0).permutation(f.shape[1])
+    r2 = oracle.vic(f[:, perm], p, 0, w.d_c, w.tau, w.n_centers)
+    np.testing.assert_allclose(r2["rho"], rho, rtol=1e-12)
+    r3 = oracle.vic(bf16(W.bf16_bits_to_f32(f) * 4.0), p, 0, w.d_c, w.tau, w.n_centers)
+    assert np.array_equal(r3["rho"], rho) and np.array_equal(r3["label"], label)
+    # near-duplicate tokens (sigma 0.01 copies) end up with their source
+    d2 = r["d2"] + np.eye(n) * 9
+    close = np.argwhere(d2 < 1e-3)
+    assert len(close) > 0
+    same = sum(label[a] == label[b] for a, b in close)
+    assert same >= 0.9 * len(close)
+
+
+def test_num_centers_ceiling():
+    assert oracle.vic_num_centers(576, 0.05) == 29       # ceil(28.8)
+    assert oracle.vic_num_centers(100, 0.05) == 5        # exact product: no spurious +1
+    assert oracle.vic_num_centers(10, 0.0) == 0
+    assert oracle.vic_num_centers(10, 2.0) == 10
+
+
+# =============================================================================== O5: compaction
+def _toy_sequence(N=23, H=3, d=8, Dh=16, seed=0):
+    rng = np.random.default_rng(seed)
+    return (rng.integers(0, 65536, (N, Dh)).astype(np.uint16), rng.integers(0, 65536, (H, N, d)).astype(np.uint16),
+            rng.integers(0, 65536, (H, N, d)).astype(np.uint16))
+
+
+def test_compact_identity_and_none():
+    hid, K, V = _toy_sequence()
+    N = hid.shape[0]
+    vs, vl = 4, 12
+    r = oracle.compact(hid, K, V, N, vs, vl, np.arange(vl), N)
+    assert r["out_len"] == N and np.array_equal(r["hidden"], hid) and np.array_equal(r["K"], K) and np.array_equal(r["V"], V)
+    assert r["kept_pos"].tolist() == list(range(N))
+    r = oracle.compact(hid, K, V, N, vs, vl, np.zeros(0, np.int32), N)
+    text = list(range(vs)) + list(range(vs + vl, N))
+    assert r["out_len"] == N - vl and r["kept_pos"][: N - vl].tolist() == text
+    assert np.array_equal(r["hidden"][: N - vl], hid[text]) and np.array_equal(r["K"][:, : N - vl], K[:, text])
+
+
+def test_compact_rows_and_order():
+    hid, K, V = _toy_sequence(seed=1)
+    N, vs, vl = hid.shape[0], 5, 10
+    keep = np.array([1, 2, 7, 9], dtype=np.int32)
+    r = oracle.compact(hid, K, V, N, vs, vl, keep, N)
+    src = list(range(vs)) + [vs + k for k in keep] + list(range(vs + vl, N))
+    L = r["out_len"]
+    assert L == len(src) and r["kept_pos"][:L].tolist() == src
+    assert np.all(np.diff(r["kept_pos"][:L]) > 0)
+    assert np.array_equal(r["hidden"][:L], hid[src]) and np.array_equal(r["V"][:, :L], V[:, src])
+    assert np.all(r["hidden"][L:] == 0)
+    # a shorter sequence inside a longer buffer: rows past seq_len are ignored
+    r2 = oracle.compact(hid, K, V, N - 3, vs, vl, keep, N)
+    assert r2["out_len"] == L - 3 and np.array_equal(r2["K"][:, : L - 3], K[:, src[:-3]])
+
+
+def test_compact_composes():
+    hid, K, V = _toy_sequence(N=40, seed=2)
+    N, vs, vl = 40, 6, 30
+    a = np.array(sorted(np.random.default_rng(0).permutation(vl)[:17]), dtype=np.int32)
+    b = np.array(sorted(np.random.default_rng(1).permutation(17)[:6]), dtype=np.int32)
+    r1 = oracle.compact(hid, K, V, N, vs, vl, a, N)
+    L1 = r1["out_len"]
+    r2 = oracle.compact(r1["hidden"], r1["K"], r1["V"], L1, vs, 17, b, N)
+    rc = oracle.compact(hid, K, V, N, vs, vl, a[b], N)
+    L = rc["out_len"]
+    assert r2["out_len"] == L
+    assert np.array_equal(r2["hidden"][:L], rc["hidden"][:L]) and np.array_equal(r2["K"][:, :L], rc["K"][:, :L])
+    assert np.array_equal(r1["kept_pos"][:L1][r2["kept_pos"][:L]], rc["kept_pos"][:L])
+
+
+# =============================================================================== schedule (Alg. 1, Eq. 10)
+def test_retention_table_counts_and_compression():
+    rows = [list(map(float, l.split())) for l in open(os.path.join(GOLDEN, "retention_ratios.txt"))
+            if l.strip() and not l.startswith("#")]
+    m = 576
+    nominal = {66.7: 192, 77.8: 128, 88.9: 64, 94.4: 32}
+    counts = {}
+    for rate, p1, p2, p3 in rows:
+        c = tuple(oracle.stage_count(m, p) for p in (p1, p2, p3))
+        counts[rate] = c
+        assert c[0] > c[1] > c[2] > 0
+        # the printed overall rate is 1 - nominal/576; Eq. 10 averaged over the 32 layers (l_s = 2, l_d = 22)
+        # reproduces it to within a few percent of the token count
+        assert abs((1 - nominal[rate] / m) * 100 - rate) < 0.06
+        cr = oracle.cr_int(p1, p2, p3, 2, 22, 32)
+        assert abs(cr - rate / 100) < 0.02
+        assert abs(cr - (1 - (p1 * 1 + p2 * 20 + p3 * 11) / 32)) < 1e-15
+    assert counts[66.7] == (288, 253, 50) and counts[88.9] == (172, 77, 15)
+    assert counts[77.8] == (230, 165, 33) and counts[94.4] == (144, 33, 6)
+
+
+def test_chain_kept_count_equals_budget():
+    # Stage III chain on the tiny workload: kept count == min(budget, n) at every step
+    w = W.workload("tiny")
+    n = w.Nv
+    for step, k in enumerate(w.budgets):
+        K, _ = W.make_kv(w, step, n)
+        s = oracle.knorm(K, w.vis_start, n)
+        for b in range(w.B):
+            keep = oracle.select_plain(s[b], k)
+            assert len(keep) == min(k, n)
+        n = min(k, n)
