@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the ViTCoP pruning operator chain on B200.
+
+One "step" = one pass of the whole hot path over one batch of the LLaVA-1.5-shaped batch-16 workload
+("c1"): redundancy filter (VIC clustering of the vision features) followed by the fused pruning step
+(K-norm -> cluster-quota selection -> compaction of hidden states, K and V).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c1]
+
+Prints ONE JSON line.  `value` is visual tokens pruned per second with the inputs resident in HBM
+(CUDA-event time per step, L2 flushed between steps); `e2e` is the same metric through the public API
+with pinned HOST buffers, host<->device copies inside the timed region.  `--impl reference` times the
+CPU oracle (test infrastructure) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_17818_b200 import workloads as W  # noqa: E402
+
+METRIC = "visual_tokens_pruned_per_s"
+UNIT = "tokens/s"
+KERNELS_PER_STEP = 8   # row_stats, gram(rho), rho_reduce, gram(delta), vic_finalize, knorm, select, compact
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------ oracle legs
+def oracle_step(w, feat, pos, K, V, hidden, budget):
+    """One step of the hot path on the CPU oracle; returns the number of visual tokens pruned."""
+    import oracle
+    B = feat.shape[0]
+    score = oracle.knorm(K, w.vis_start, w.Nv)
+    pruned = 0
+    for b in range(B):
+        r = oracle.vic(feat[b], pos[b], 0, w.d_c, w.tau, w.n_centers)
+        keep, _, _ = oracle.select_quota(score[b], r["label"], budget)
+        oracle.compact(hidden[b], K[b], V[b], w.N, w.vis_start, w.Nv, keep, w.T + budget)
+        pruned += w.Nv - len(keep)
+    return pruned
+
+
+def time_oracle(w, steps, warmup, sample_B):
+    import oracle
+    feat, pos = W.make_features(w, B=sample_B), W.make_positions(w)[:sample_B]
+    K, V = W.make_kv(w, 0, w.Nv, B=sample_B)
+    hidden = W.make_hidden(w, B=sample_B)
+    oracle.build()
+    for _ in range(warmup):
+        oracle_step(w, feat, pos, K, V, hidden, w.budgets[0])
+    t0 = time.perf_counter()
+    pruned = 0
+    for _ in range(steps):
+        pruned += oracle_step(w, feat, pos, K, V, hidden, w.budgets[0])
+    dt = time.perf_counter() - t0
+    return pruned / dt, dt / steps, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = W.workload(args.workload)
+    sample_B = min(w.B, 4)
+    value, sec_per_step, cores = time_oracle(w, args.steps, args.warmup, sample_B)
+    sample = f"{sample_B} of {w.B} samples of workload {w.name} per step (fp64 CPU oracle, whole hot path)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
+                   "budget": w.budgets[0], "n_centers": w.n_centers},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.sm, self.reasons, self.sm_max = [], set(), None
+        self._stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.sm.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop.set()
+        self.join(timeout=2)
+        return {"sm_mhz": (float(np.median(self.sm)) if self.sm else None), "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+class Step:
+    """Device buffers and the two API calls of one hot-path step."""
+
+    def __init__(self, w, torch, vb, dev):
+        self.w, self.torch, self.vb = w, torch, vb
+        B, n = w.B, w.Nv
+        self.budget = w.budgets[0]
+        self.Ncap = w.T + self.budget
+        e = lambda *s, dt=torch.bfloat16: torch.empty(s, dtype=dt, device=dev)
+        self.feat, self.pos = e(B, n, w.D), e(B, n, 2, dt=torch.float32)
+        self.K, self.V, self.hidden = e(B, w.H, w.N, w.d), e(B, w.H, w.N, w.d), e(B, w.N, w.Dh)
+        self.label, self.ncl = e(B, n, dt=torch.int32), e(B, dt=torch.int32)
+        self.ho, self.Ko, self.Vo = e(B, self.Ncap, w.Dh), e(B, w.H, self.Ncap, w.d), e(B, w.H, self.Ncap, w.d)
+        self.olen, self.nkeep = e(B, dt=torch.int32), e(B, dt=torch.int32)
+        self.kpos = e(B, self.Ncap, dt=torch.int32)
+        self.ws_f = vb.alloc_workspace(vb.OP_FILTER, device=dev, B=B, Nv=n, D=w.D)
+        self.ws_s = vb.alloc_workspace(vb.OP_PRUNE_STEP, device=dev, B=B, Nv=n)
+
+    def upload(self, host, non_blocking=True):
+        for name in ("feat", "pos", "K", "V", "hidden"):
+            getattr(self, name).copy_(host[name], non_blocking=non_blocking)
+
+    def filter(self):
+        w = self.w
+        self.vb.vitcop_redundancy_filter(self.feat, self.pos, self.label, self.ncl, self.ws_f, metric=0, d_c=w.d_c,
+                                         tau=w.tau, n_centers=w.n_centers)
+
+    def prune(self):
+        w = self.w
+        self.vb.vitcop_prune_step(self.hidden, self.K, self.V, w.vis_start, w.Nv, w.Nv, self.budget, self.ho, self.Ko,
+                                  self.Vo, self.olen, self.ws_s, label=self.label, kept_pos=self.kpos,
+                                  n_keep_out=self.nkeep)
+
+    def run(self):
+        self.filter()
+        self.prune()
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_17818_b200 import binding as vb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    vb.lib()                                   # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w = W.workload(args.workload)
+    peaks = measured_peaks()
+
+    # host inputs (pinned) ---------------------------------------------------------------------------
+    feat_b, pos = W.make_features(w), W.make_positions(w)
+    K_b, V_b = W.make_kv(w, 0, w.Nv)
+    hid_b = W.make_hidden(w)
+    host = {"feat": torch.from_numpy(feat_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
+            "pos": torch.from_numpy(pos).pin_memory(),
+            "K": torch.from_numpy(K_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
+            "V": torch.from_numpy(V_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
+            "hidden": torch.from_numpy(hid_b.view(np.int16)).view(torch.bfloat16).pin_memory()}
+    st = Step(w, torch, vb, dev)
+    st.upload(host, non_blocking=False)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)     # > 4x the 126 MB L2
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        """Per-step CUDA-event times (ms) with an L2 flush before every step."""
+        for _ in range(warmup):
+            flush.zero_()
+            fn()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in evs:
+            flush.zero_()
+            a.record()
+            fn()
+            b.record()
+        barrier()
+        return np.array([a.elapsed_time(b) for a, b in evs], dtype=np.float64)
+
+    # whole step, device resident ------------------------------------------------------------------------
+    sampler = ClockSampler(local)
+    sampler.start()
+    t_step = timed(st.run, args.steps, args.warmup)
+    clocks = sampler.stop()
+    n_keep = st.nkeep.cpu().numpy()
+    pruned_per_step = int((w.Nv - n_keep).sum())
+    total_ms = float(t_step.sum())
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * pruned_per_step * args.steps / (total_ms * 1e-3)
+
+    # per-stage times (same protocol) ------------------------------------------------------------------
+    stage = {}
+    score = torch.empty((w.B, w.Nv), dtype=torch.float32, device=dev)
+    kidx = torch.empty((w.B, w.Nv), dtype=torch.int32, device=dev)
+    ws_sel = vb.alloc_workspace(vb.OP_SELECT, device=dev, B=w.B, Nv=w.Nv)
+    stage_fns = {
+        "filter": st.filter,
+        "knorm": lambda: vb.vitcop_knorm_score(st.K, w.vis_start, w.Nv, score),
+        "select": lambda: vb.vitcop_select(score, w.Nv, st.budget, kidx, st.nkeep, ws_sel, label=st.label),
+        "compact": lambda: vb.vitcop_compact_kv(st.hidden, st.K, st.V, w.vis_start, w.Nv, kidx, st.nkeep, st.ho,
+                                                st.Ko, st.Vo, st.olen, kept_pos=st.kpos),
+        "prune_step": st.prune,
+    }
+    n_stage = max(10, min(args.steps, 50))
+    for name, fn in stage_fns.items():
+        t = timed(fn, n_stage, 3)
+        stage[name] = {"us_median": float(np.median(t) * 1e3), "us_min": float(t.min() * 1e3)}
+    nk_total = int(st.nkeep.cpu().numpy().sum())
+    knorm_bytes = w.B * w.H * w.Nv * w.d * 2 + w.B * w.Nv * 4
+    rows_out = w.B * w.T + nk_total
+    compact_bytes = 2 * rows_out * (w.Dh + 2 * w.H * w.d) * 2
+    gram_flop = w.B * w.Nv * (w.Nv + 1) * w.D            # algorithmic: symmetric half incl. diagonal
+    stage["knorm"].update(bytes=knorm_bytes, gbs=knorm_bytes / (stage["knorm"]["us_median"] * 1e-6) / 1e9)
+    stage["compact"].update(bytes=compact_bytes, gbs=compact_bytes / (stage["compact"]["us_median"] * 1e-6) / 1e9)
+    stage["filter"].update(algorithmic_flop=gram_flop,
+                           tflops=gram_flop / (stage["filter"]["us_median"] * 1e-6) / 1e12)
+    for k in ("knorm", "compact"):
+        stage[k]["frac_of_measured_hbm"] = stage[k]["gbs"] / peaks["hbm_gbs"]
+    # the dominant single kernel of the step
+    single = {"knorm": stage["knorm"]["us_median"], "compact": stage["compact"]["us_median"]}
+    dom = max(single, key=single.get)
+    roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": stage[dom]["gbs"], "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": stage[dom]["gbs"] / peaks["hbm_gbs"], "traffic": None,
+                "peak_source": peaks["source"], "algorithmic_bytes_per_launch": stage[dom]["bytes"]}
+
+    # end to end through the public API with host buffers ----------------------------------------------------
+    out_host = {"ho": torch.empty(st.ho.shape, dtype=st.ho.dtype).pin_memory(),
+                "Ko": torch.empty(st.Ko.shape, dtype=st.Ko.dtype).pin_memory(),
+                "Vo": torch.empty(st.Vo.shape, dtype=st.Vo.dtype).pin_memory(),
+                "olen": torch.empty(st.olen.shape, dtype=st.olen.dtype).pin_memory(),
+                "kpos": torch.empty(st.kpos.shape, dtype=st.kpos.dtype).pin_memory()}
+
+    def e2e_step():
+        st.upload(host)
+        st.run()
+        out_host["ho"].copy_(st.ho, non_blocking=True)
+        out_host["Ko"].copy_(st.Ko, non_blocking=True)
+        out_host["Vo"].copy_(st.Vo, non_blocking=True)
+        out_host["olen"].copy_(st.olen, non_blocking=True)
+        out_host["kpos"].copy_(st.kpos, non_blocking=True)
+
+    n_e2e = max(5, min(args.steps, 20))
+    t_e2e = timed(e2e_step, n_e2e, 3)
+    e2e_ms = float(t_e2e.sum())
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(int(v.numel() * v.element_size()) for v in host.values())
+    d2h = sum(int(v.numel() * v.element_size()) for v in out_host.values())
+    e2e = {"value": world * pruned_per_step * n_e2e / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / n_e2e}
+
+    # CPU oracle beside it (rank 0, N = 1 only; bounded sample) ------------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample_B = min(w.B, 4)
+        v, sec, cores = time_oracle(w, 3, 1, sample_B)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{sample_B} of {w.B} samples of workload {w.name}, 3 timed passes of the whole hot path "
+                         f"({sec:.2f} s each)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, fp32 arithmetic", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
+                       "budget": st.budget, "n_centers": w.n_centers, "mode": "filter + quota prune step",
+                       "tokens_pruned_per_step": pruned_per_step, "tokens_kept_per_step": nk_total,
+                       "l2": "flushed (512 MiB memset) before every timed step", "sharding": "replicas only"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "stages": stage,
+            "us_per_step_median": float(np.median(t_step) * 1e3),
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,241 @@
+// Public C ABI of libvitcop: argument validation, workspace carving and dispatch to the launchers.
+#include <cmath>
+#include <cstdint>
+
+#include "internal.cuh"
+
+namespace vitcop {
+
+static thread_local int g_last_cuda_error = 0;
+
+int record_cuda(cudaError_t e) {
+    if (e == cudaSuccess) return VITCOP_OK;
+    g_last_cuda_error = static_cast<int>(e);
+    return VITCOP_ERR_CUDA;
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+inline bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + nb && y < x + na;
+}
+
+// Workspace of the fused step: status | score [B,Nv] | keep_idx [B,Nv] | n_keep [B]
+struct StepWs {
+    size_t off_score, off_keep, off_nkeep, total;
+    StepWs(int B, int Nv) {
+        size_t o = kStatusBytes;
+        off_score = o; o += align_up((size_t)B * Nv * sizeof(float), 256);
+        off_keep = o;  o += align_up((size_t)B * Nv * sizeof(int32_t), 256);
+        off_nkeep = o; o += align_up((size_t)B * sizeof(int32_t), 256);
+        total = o;
+    }
+};
+
+int reset_status(void* ws, cudaStream_t s) { return record_cuda(cudaMemsetAsync(ws, 0, kStatusBytes, s)); }
+
+int check_span(int N, int vis_start, const int32_t* vis_len, int vis_len_uniform, int Nv_cap) {
+    if (vis_start < 0 || vis_start > N) return VITCOP_ERR_INVALID_ARG;
+    if (!vis_len) {
+        if (vis_len_uniform < 0 || vis_start + (int64_t)vis_len_uniform > N) return VITCOP_ERR_INVALID_ARG;
+        if (Nv_cap >= 0 && vis_len_uniform > Nv_cap) return VITCOP_ERR_INVALID_ARG;
+    } else if (Nv_cap >= 0 && vis_start + (int64_t)Nv_cap > N) {
+        // device-side lengths are clamped to the capacity, which itself must fit the sequence
+        return VITCOP_ERR_INVALID_ARG;
+    }
+    return VITCOP_OK;
+}
+
+}  // namespace
+}  // namespace vitcop
+
+using namespace vitcop;
+
+extern "C" {
+
+const char* vitcop_status_string(int status) {
+    switch (status) {
+        case VITCOP_OK: return "ok";
+        case VITCOP_ERR_INVALID_ARG: return "invalid argument";
+        case VITCOP_ERR_UNSUPPORTED: return "unsupported shape or alignment";
+        case VITCOP_ERR_WORKSPACE: return "workspace missing or too small";
+        case VITCOP_ERR_BUDGET: return "budget smaller than the number of clusters";
+        case VITCOP_ERR_CUDA: return "CUDA runtime error";
+        case VITCOP_ERR_TIMEOUT: return "bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+int vitcop_last_cuda_error(void) { return g_last_cuda_error; }
+
+int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, int Dh, size_t* bytes) {
+    (void)H; (void)N; (void)d; (void)Dh;
+    if (!bytes || B < 0 || Nv < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
+    switch (op) {
+        case VITCOP_OP_FILTER: *bytes = filter_workspace_bytes(B, Nv, D); return VITCOP_OK;
+        case VITCOP_OP_SIMILARITY: *bytes = similarity_workspace_bytes(B, Nv, D); return VITCOP_OK;
+        case VITCOP_OP_KNORM: *bytes = 0; return VITCOP_OK;
+        case VITCOP_OP_COMPACT: *bytes = 0; return VITCOP_OK;
+        case VITCOP_OP_SELECT: *bytes = kStatusBytes; return VITCOP_OK;
+        case VITCOP_OP_PRUNE_STEP: *bytes = StepWs(B, Nv).total; return VITCOP_OK;
+        default: return VITCOP_ERR_INVALID_ARG;
+    }
+}
+
+int vitcop_poll_status(const void* workspace, void* stream, int* device_status) {
+    if (!workspace || !device_status) return VITCOP_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    int rc = record_cuda(cudaMemcpyAsync(&v, workspace, sizeof(int), cudaMemcpyDeviceToHost, s));
+    if (rc != VITCOP_OK) return rc;
+    rc = record_cuda(cudaStreamSynchronize(s));
+    if (rc != VITCOP_OK) return rc;
+    *device_status = v;
+    return VITCOP_OK;
+}
+
+int vitcop_knorm_score(const void* K, int B, int H, int N, int d, int64_t stride_b, int64_t stride_h,
+                       int64_t stride_n, int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score,
+                       int Nv_cap, void* stream) {
+    if (!K || !score || B < 0 || H < 0 || N < 0 || d < 0 || Nv_cap < 0) return VITCOP_ERR_INVALID_ARG;
+    if (stride_b < 0 || stride_h < 0 || stride_n < 0) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_span(N, vis_start, vis_len, vis_len_uniform, Nv_cap);
+    if (rc != VITCOP_OK) return rc;
+    if (d % 8 || stride_b % 8 || stride_h % 8 || stride_n % 8 || !aligned16(K)) return VITCOP_ERR_UNSUPPORTED;
+    if (B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    return launch_knorm(K, B, H, d, stride_b, stride_h, stride_n, vis_start, vis_len, vis_len_uniform, score, Nv_cap,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int vitcop_select(const float* score, const int32_t* label, int B, const int32_t* vis_len, int vis_len_uniform,
+                  int Nv_cap, const vitcop_select_params* p, int32_t* keep_idx, int keep_stride, int32_t* n_keep,
+                  uint8_t* keep_mask, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!score || !p || !keep_idx || !n_keep || B < 0 || Nv_cap < 0 || keep_stride < 0) return VITCOP_ERR_INVALID_ARG;
+    if (p->mode != 0 && p->mode != 1) return VITCOP_ERR_INVALID_ARG;
+    if (p->budget < 0) return VITCOP_ERR_INVALID_ARG;
+    if (p->mode == 1 && !label) return VITCOP_ERR_INVALID_ARG;
+    if (!vis_len && (vis_len_uniform < 0 || vis_len_uniform > Nv_cap)) return VITCOP_ERR_INVALID_ARG;
+    if (keep_stride < (p->budget < Nv_cap ? p->budget : Nv_cap)) return VITCOP_ERR_INVALID_ARG;
+    if (Nv_cap > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < kStatusBytes) return VITCOP_ERR_WORKSPACE;
+    if (!aligned256(workspace)) return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    return launch_select(score, label, B, vis_len, vis_len_uniform, Nv_cap, p->mode, p->largest ? 1 : 0, p->budget,
+                         keep_idx, keep_stride, n_keep, keep_mask, static_cast<int*>(workspace), s, false);
+}
+
+static int check_compact_args(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                              int vis_start, const int32_t* vis_len, int vis_len_uniform, void* hidden_out,
+                              void* K_out, void* V_out, int Ncap) {
+    if (B < 0 || H < 0 || N < 0 || d < 0 || Dh < 0 || Ncap < 0) return VITCOP_ERR_INVALID_ARG;
+    if ((hidden == nullptr) != (hidden_out == nullptr)) return VITCOP_ERR_INVALID_ARG;
+    if ((K == nullptr) != (K_out == nullptr)) return VITCOP_ERR_INVALID_ARG;
+    if ((V == nullptr) != (V_out == nullptr)) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_span(N, vis_start, vis_len, vis_len_uniform, -1);
+    if (rc != VITCOP_OK) return rc;
+    if (d % 8 || Dh % 8) return VITCOP_ERR_UNSUPPORTED;
+    if (!aligned16(hidden) || !aligned16(K) || !aligned16(V) || !aligned16(hidden_out) || !aligned16(K_out) ||
+        !aligned16(V_out))
+        return VITCOP_ERR_UNSUPPORTED;
+    if (B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    const size_t hin = (size_t)B * N * Dh * 2, hout = (size_t)B * Ncap * Dh * 2;
+    const size_t kin = (size_t)B * H * N * d * 2, kout = (size_t)B * H * Ncap * d * 2;
+    const void* ins[3] = {hidden, K, V};
+    const size_t insz[3] = {hin, kin, kin};
+    const void* outs[3] = {hidden_out, K_out, V_out};
+    const size_t outsz[3] = {hout, kout, kout};
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j)
+            if (overlaps(ins[i], insz[i], outs[j], outsz[j])) return VITCOP_ERR_INVALID_ARG;
+    return VITCOP_OK;
+}
+
+int vitcop_compact_kv(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                      const int32_t* seq_len, int vis_start, const int32_t* vis_len, int vis_len_uniform,
+                      const int32_t* keep_idx, int keep_stride, const int32_t* n_keep, void* hidden_out, void* K_out,
+                      void* V_out, int Ncap, int32_t* kept_pos, int32_t* out_len, void* stream) {
+    if (!keep_idx || !n_keep || !out_len || keep_stride < 0) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_compact_args(hidden, K, V, B, H, N, d, Dh, vis_start, vis_len, vis_len_uniform, hidden_out, K_out,
+                                V_out, Ncap);
+    if (rc != VITCOP_OK) return rc;
+    return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
+                          keep_stride, n_keep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len,
+                          static_cast<cudaStream_t>(stream), false);
+}
+
+int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                      const int32_t* seq_len, int vis_start, const int32_t* vis_len, int vis_len_uniform, int Nv_cap,
+                      const int32_t* label, int budget, void* hidden_out, void* K_out, void* V_out, int Ncap,
+                      int32_t* kept_pos, int32_t* out_len, float* score_out, int32_t* keep_idx_out,
+                      int32_t* n_keep_out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!K || !out_len || budget < 0 || Nv_cap < 0) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_compact_args(hidden, K, V, B, H, N, d, Dh, vis_start, vis_len, vis_len_uniform, hidden_out, K_out,
+                                V_out, Ncap);
+    if (rc != VITCOP_OK) return rc;
+    rc = check_span(N, vis_start, vis_len, vis_len_uniform, Nv_cap);
+    if (rc != VITCOP_OK) return rc;
+    if (Nv_cap > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
+    const StepWs lay(B, Nv_cap);
+    if (!workspace || workspace_bytes < lay.total || !aligned256(workspace)) return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    float* score = score_out ? score_out : reinterpret_cast<float*>(ws + lay.off_score);
+    int32_t* keep = keep_idx_out ? keep_idx_out : reinterpret_cast<int32_t*>(ws + lay.off_keep);
+    int32_t* nkeep = n_keep_out ? n_keep_out : reinterpret_cast<int32_t*>(ws + lay.off_nkeep);
+    rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    rc = launch_knorm(K, B, H, d, (int64_t)H * N * d, (int64_t)N * d, d, vis_start, vis_len, vis_len_uniform, score,
+                      Nv_cap, s);
+    if (rc != VITCOP_OK) return rc;
+    rc = launch_select(score, label, B, vis_len, vis_len_uniform, Nv_cap, label ? 1 : 0, 0, budget, keep, Nv_cap,
+                       nkeep, nullptr, reinterpret_cast<int*>(ws), s, true);
+    if (rc != VITCOP_OK) return rc;
+    return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep, Nv_cap,
+                          nkeep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, s, true);
+}
+
+int vitcop_redundancy_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params* p,
+                             int32_t* label, int32_t* n_clusters, float* rho, float* delta2, int32_t* parent,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (!feat || !p || !label || !n_clusters || B < 0 || n < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
+    if (p->metric != 0 && p->metric != 1) return VITCOP_ERR_INVALID_ARG;
+    if (!(p->d_c > 0.f)) return VITCOP_ERR_INVALID_ARG;
+    if (D % 64 || !aligned16(feat) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < filter_workspace_bytes(B, n, D) || !aligned256(workspace))
+        return VITCOP_ERR_WORKSPACE;
+    int nc = p->n_centers;
+    if (nc <= 0) {
+        const double v = std::ceil((double)n * (double)p->alpha);
+        nc = v < 0 ? 0 : (v > n ? n : (int)v);
+    }
+    if (nc > n) nc = n;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    if (B == 0 || n == 0) return VITCOP_OK;
+    return launch_filter(feat, pos, B, n, D, *p, nc, label, n_clusters, rho, delta2, parent, workspace, s);
+}
+
+int vitcop_similarity_rows(const void* feat, int B, int n, int D, int metric, int row_begin, int row_end, float* out,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    if (!feat || !out || B < 0 || n < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
+    if (metric != 0 && metric != 1) return VITCOP_ERR_INVALID_ARG;
+    if (row_begin < 0 || row_end < row_begin || row_end > n) return VITCOP_ERR_INVALID_ARG;
+    if (D % 64 || !aligned16(feat) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < similarity_workspace_bytes(B, n, D) || !aligned256(workspace))
+        return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    if (B == 0 || n == 0 || row_end == row_begin) return VITCOP_OK;
+    return launch_similarity_rows(feat, B, n, D, metric, row_begin, row_end, out, workspace, s);
+}
+
+}  // extern "C"

@@ -1,0 +1,146 @@
+// Order-preserving compaction of hidden states and the K/V cache (bit-exact row gather).
+//
+// One CTA per (output row, sample).  The source position of the row comes from the ascending
+// keep list; the CTA then moves the hidden row and the row of every K and V head with 128-bit
+// loads that are all issued before the first store, so that each thread keeps several
+// independent 16-byte requests in flight.  Dropped rows are never read.
+#include "internal.cuh"
+
+namespace vitcop {
+namespace {
+
+constexpr int kCompactThreads = 256;
+constexpr int kChunk = 8;   // 16-byte pieces a thread holds in registers at once
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+
+// Piece q of the row: [0, dh8) hidden, then H*d8 pieces of K (head-major), then H*d8 pieces of V.
+struct RowMap {
+    const uint4 *hid, *K, *V;
+    uint4 *hid_o, *K_o, *V_o;
+    int dh8, d8, hd8;              // pieces per hidden row, per head row, per all heads
+    int64_t k_head_in, k_head_out;  // pieces between consecutive heads (N*d8, Ncap*d8)
+    __device__ __forceinline__ void locate(int q, const uint4*& src, uint4*& dst) const {
+        if (q < dh8) {
+            src = hid + q;
+            dst = hid_o + q;
+        } else {
+            q -= dh8;
+            const bool isv = q >= hd8;
+            if (isv) q -= hd8;
+            const int h = q / d8, e = q - h * d8;
+            src = (isv ? V : K) + h * k_head_in + e;
+            dst = (isv ? V_o : K_o) + h * k_head_out + e;
+        }
+    }
+};
+
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, const uint4* __restrict__ V, int H, int N,
+               int d8, int dh8, const int32_t* __restrict__ seq_len, int vis_start,
+               const int32_t* __restrict__ vis_len, int vis_len_uniform, const int32_t* __restrict__ keep_idx,
+               int keep_stride, const int32_t* __restrict__ n_keep, uint4* __restrict__ hidden_out,
+               uint4* __restrict__ K_out, uint4* __restrict__ V_out, int Ncap, int32_t* __restrict__ kept_pos,
+               int32_t* __restrict__ out_len) {
+    grid_dependency_wait();
+    const int b = blockIdx.y;
+    const int r = blockIdx.x;
+    const int L = seq_len ? min(seq_len[b], N) : N;
+    int nv = vis_len ? vis_len[b] : vis_len_uniform;
+    nv = max(0, min(nv, L - vis_start));
+    const int nk = max(0, min(n_keep[b], nv));
+    const int olen = L - nv + nk;
+    if (r == 0 && threadIdx.x == 0) out_len[b] = olen;
+    if (r >= Ncap) return;
+    if (r >= olen) {
+        if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = -1;
+        return;
+    }
+    int src_row;
+    if (r < vis_start) src_row = r;
+    else if (r < vis_start + nk) {
+        int ki = keep_idx[(int64_t)b * keep_stride + (r - vis_start)];
+        ki = max(0, min(ki, nv - 1));                     // a corrupt index can never leave the span
+        src_row = vis_start + ki;
+    } else src_row = r - nk + nv;
+    if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = src_row;
+
+    RowMap m;
+    m.dh8 = hidden ? dh8 : 0;
+    m.d8 = d8 > 0 ? d8 : 1;
+    m.hd8 = H * d8;
+    m.k_head_in = (int64_t)N * d8;
+    m.k_head_out = (int64_t)Ncap * d8;
+    m.hid = hidden ? hidden + ((int64_t)b * N + src_row) * dh8 : nullptr;
+    m.hid_o = hidden ? hidden_out + ((int64_t)b * Ncap + r) * dh8 : nullptr;
+    m.K = K ? K + ((int64_t)b * H * N + src_row) * d8 : nullptr;
+    m.K_o = K ? K_out + ((int64_t)b * H * Ncap + r) * d8 : nullptr;
+    m.V = V ? V + ((int64_t)b * H * N + src_row) * d8 : nullptr;
+    m.V_o = V ? V_out + ((int64_t)b * H * Ncap + r) * d8 : nullptr;
+    // K absent but V present: shift V into K's slot range
+    int total = m.dh8;
+    if (K && V) total += 2 * m.hd8;
+    else if (K) total += m.hd8;
+    else if (V) {
+        m.K = m.V;
+        m.K_o = m.V_o;
+        total += m.hd8;
+    }
+
+    for (int q0 = threadIdx.x; q0 < total; q0 += kCompactThreads * kChunk) {
+        uint4 v[kChunk];
+        uint4* dst[kChunk];
+#pragma unroll
+        for (int u = 0; u < kChunk; ++u) {
+            const int q = q0 + u * kCompactThreads;
+            dst[u] = nullptr;
+            if (q < total) {
+                const uint4* src;
+                m.locate(q, src, dst[u]);
+                v[u] = ld_stream(src);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kChunk; ++u)
+            if (dst[u]) st_stream(dst[u], v[u]);
+    }
+    grid_dependency_launch_dependents();
+}
+
+}  // namespace
+
+int launch_compact(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                   const int32_t* seq_len, int vis_start, const int32_t* vis_len, int vis_len_uniform,
+                   const int32_t* keep_idx, int keep_stride, const int32_t* n_keep, void* hidden_out, void* K_out,
+                   void* V_out, int Ncap, int32_t* kept_pos, int32_t* out_len, cudaStream_t stream, bool pdl) {
+    if (B <= 0) return VITCOP_OK;
+    cudaLaunchConfig_t cfg = {};
+    // rows past min(N, Ncap) cannot exist; one extra CTA row keeps out_len written when Ncap == 0
+    const int rows = Ncap > 0 ? Ncap : 1;
+    cfg.gridDim = dim3(rows, B);
+    cfg.blockDim = dim3(kCompactThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return record_cuda(cudaLaunchKernelEx(
+        &cfg, compact_kernel, static_cast<const uint4*>(hidden), static_cast<const uint4*>(K),
+        static_cast<const uint4*>(V), H, N, d / 8, Dh / 8, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
+        keep_stride, n_keep, static_cast<uint4*>(hidden_out), static_cast<uint4*>(K_out), static_cast<uint4*>(V_out),
+        Ncap, kept_pos, out_len));
+}
+
+}  // namespace vitcop

@@ -1,0 +1,54 @@
+// Internal declarations shared by the translation units of libvitcop (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vitcop.h"
+
+namespace vitcop {
+
+// Device status word lives in the first 256 bytes of every workspace.
+constexpr size_t kStatusBytes = 256;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Records the first failing CUDA runtime error of the calling thread.
+int record_cuda(cudaError_t e);
+
+// ---- launchers (enqueue on `stream`, return VITCOP_OK or VITCOP_ERR_CUDA) -------------------------
+int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
+                 int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
+                 cudaStream_t stream);
+
+int launch_select(const float* score, const int32_t* label, int B, const int32_t* vis_len, int vis_len_uniform,
+                  int Nv_cap, int mode, int largest, int budget, int32_t* keep_idx, int keep_stride,
+                  int32_t* n_keep, uint8_t* keep_mask, int* status_word, cudaStream_t stream, bool pdl);
+
+int launch_compact(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                   const int32_t* seq_len, int vis_start, const int32_t* vis_len, int vis_len_uniform,
+                   const int32_t* keep_idx, int keep_stride, const int32_t* n_keep, void* hidden_out, void* K_out,
+                   void* V_out, int Ncap, int32_t* kept_pos, int32_t* out_len, cudaStream_t stream, bool pdl);
+
+size_t filter_workspace_bytes(int B, int n, int D);
+size_t similarity_workspace_bytes(int B, int n, int D);
+int launch_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params& p,
+                  int n_centers, int32_t* label, int32_t* n_clusters, float* rho, float* delta2, int32_t* parent,
+                  void* workspace, cudaStream_t stream);
+int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, int row_begin, int row_end,
+                           float* out, void* workspace, cudaStream_t stream);
+
+// ---- small device helpers ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// Programmatic dependent launch: wait until the preceding kernel on the stream has completed
+// (no-op when the kernel was not launched with the PDL attribute).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
+}  // namespace vitcop

@@ -1,0 +1,96 @@
+// K-norm saliency (Eq. 4): score_i = sqrt( sum_h sum_e K[b,h,i,e]^2 ) over the visual span.
+//
+// HBM-bound streaming reduction.  A group of LPR consecutive lanes owns one token: every lane
+// issues 128-bit loads (8 bf16) from the token's row in each head, squares in fp32 (a bf16
+// product is exact in fp32), accumulates over heads in registers and the group finishes with
+// xor-shuffles.  Consecutive tokens of one head are contiguous in memory, so a CTA's loads of one
+// head form one contiguous run of TOKENS_PER_CTA * d * 2 bytes.
+#include "internal.cuh"
+
+namespace vitcop {
+namespace {
+
+constexpr int kKnormThreads = 128;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void sq_acc(const uint4& v, float& a0, float& a1) {
+    float x;
+    x = bf16lo(v.x); a0 = fmaf(x, x, a0);
+    x = bf16hi(v.x); a1 = fmaf(x, x, a1);
+    x = bf16lo(v.y); a0 = fmaf(x, x, a0);
+    x = bf16hi(v.y); a1 = fmaf(x, x, a1);
+    x = bf16lo(v.z); a0 = fmaf(x, x, a0);
+    x = bf16hi(v.z); a1 = fmaf(x, x, a1);
+    x = bf16lo(v.w); a0 = fmaf(x, x, a0);
+    x = bf16hi(v.w); a1 = fmaf(x, x, a1);
+}
+
+// Strides are in units of 16 bytes (8 elements).
+template <int LPR, int UNROLL>
+__global__ void __launch_bounds__(kKnormThreads)
+knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh, int64_t sn, int vis_start,
+             const int32_t* __restrict__ vis_len, int vis_len_uniform, float* __restrict__ score, int Nv_cap) {
+    grid_dependency_wait();
+    const int b = blockIdx.y;
+    const int nv = vis_len ? vis_len[b] : vis_len_uniform;
+    constexpr int kTok = kKnormThreads / LPR;
+    const int sub = threadIdx.x % LPR;
+    const int i = blockIdx.x * kTok + threadIdx.x / LPR;
+    float a0 = 0.f, a1 = 0.f;
+    if (i < nv) {
+        const uint4* base = K + b * sb + (int64_t)(vis_start + i) * sn;
+        for (int c = sub; c < d8; c += LPR) {
+            const uint4* p = base + c;
+            int h = 0;
+            for (; h + UNROLL <= H; h += UNROLL) {
+                uint4 v[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(p + (int64_t)(h + u) * sh);
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) sq_acc(v[u], a0, a1);
+            }
+            for (; h < H; ++h) {
+                const uint4 v = ld_stream(p + (int64_t)h * sh);
+                sq_acc(v, a0, a1);
+            }
+        }
+    }
+    float acc = a0 + a1;
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (i < nv && sub == 0) score[(int64_t)b * Nv_cap + i] = sqrtf(acc);
+    grid_dependency_launch_dependents();
+}
+
+}  // namespace
+
+int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
+                 int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
+                 cudaStream_t stream) {
+    if (B <= 0 || Nv_cap <= 0 || H <= 0) return VITCOP_OK;
+    const int d8 = d / 8;
+    const int span = vis_len ? Nv_cap : vis_len_uniform;
+    if (span <= 0) return VITCOP_OK;
+    const uint4* Kp = static_cast<const uint4*>(K);
+    const int64_t sb = stride_b / 8, sh = stride_h / 8, sn = stride_n / 8;
+    auto go = [&](auto kern, int lpr) {
+        const int tok = kKnormThreads / lpr;
+        dim3 grid((span + tok - 1) / tok, B);
+        kern<<<grid, kKnormThreads, 0, stream>>>(Kp, H, d8, sb, sh, sn, vis_start, vis_len, vis_len_uniform, score,
+                                                  Nv_cap);
+    };
+    if (d8 >= 16) go(knorm_kernel<16, 8>, 16);
+    else if (d8 >= 8) go(knorm_kernel<8, 8>, 8);
+    else if (d8 >= 4) go(knorm_kernel<4, 8>, 4);
+    else go(knorm_kernel<1, 8>, 1);
+    return record_cuda(cudaGetLastError());
+}
+
+}  // namespace vitcop

@@ -1,0 +1,193 @@
+"""Shared plumbing of the GPU parity tests: upload seeded inputs, call the C ABI through the binding,
+run the CPU oracle on the same bits and compare under the stated tolerances."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2601_17818_b200 import binding as vb
+from paper_2601_17818_b200 import workloads as W
+
+# Tolerances (written out here so that the tests read as the contract):
+KNORM_RTOL = 1e-5        # K-norm: |gpu - oracle| <= 1e-5 * oracle
+SIM_ATOL = 1e-5          # cosine similarity in [-1, 1]: absolute 1e-5
+GRAM_RTOL = 1e-5         # raw Gram (euclid): |gpu - oracle| <= 1e-5 * sqrt(g_ii * g_jj)
+RHO_RTOL = 1e-5          # density
+D2_ATOL, D2_RTOL = 2e-5, 1e-5   # delta^2 (2 - 2s cancels for near-duplicates, hence the absolute part)
+VIC_TOLS = dict(tol_rho=RHO_RTOL, tol_d2_abs=D2_ATOL, tol_d2_rel=D2_RTOL, tol_sp=1e-6)
+
+DEV = "cuda"
+
+
+def dev_i32(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(DEV)
+
+
+def gpu_knorm(K_bits, vis_start, vis_len, Nv_cap=None):
+    K = vb.bf16_tensor(K_bits)
+    B = K.shape[0]
+    if np.isscalar(vis_len):
+        cap = int(vis_len) if Nv_cap is None else Nv_cap
+        vl = int(vis_len)
+    else:
+        cap = int(max(vis_len)) if Nv_cap is None else Nv_cap
+        vl = dev_i32(vis_len)
+    score = torch.full((B, max(cap, 1)), -7.0, dtype=torch.float32, device=DEV)
+    vb.vitcop_knorm_score(K, vis_start, vl, score)
+    torch.cuda.synchronize()
+    return score.cpu().numpy()[:, :cap]
+
+
+def gpu_select(score, budget, vis_len=None, label=None, largest=False, want_mask=True):
+    s = torch.from_numpy(np.ascontiguousarray(score, dtype=np.float32)).to(DEV)
+    B, cap = s.shape
+    vl = cap if vis_len is None else (int(vis_len) if np.isscalar(vis_len) else dev_i32(vis_len))
+    stride = max(1, min(budget, cap))
+    keep = torch.full((B, stride), -9, dtype=torch.int32, device=DEV)
+    nk = torch.full((B,), -9, dtype=torch.int32, device=DEV)
+    mask = torch.full((B, cap), 7, dtype=torch.uint8, device=DEV) if want_mask else None
+    ws = vb.alloc_workspace(vb.OP_SELECT, B=B, Nv=cap)
+    lab = None if label is None else dev_i32(label)
+    vb.vitcop_select(s, vl, budget, keep, nk, ws, label=lab, largest=largest, keep_mask=mask)
+    status = vb.vitcop_poll_status(ws)
+    nk = nk.cpu().numpy()
+    keep = keep.cpu().numpy()
+    return [keep[b, :max(nk[b], 0)] for b in range(B)], nk, (None if mask is None else mask.cpu().numpy()), status
+
+
+def oracle_band_check(score64, gpu_keep, k, rtol, largest=False):
+    """Kept-set comparison with the tolerance band at the cut (plain top-k of one sequence).
+
+    Tokens whose oracle score lies within `rtol` (relative) of the cut may go either way; every other
+    token must agree with the oracle, and the kept count must be exact."""
+    n = len(score64)
+    want = oracle.select_plain(score64, k, largest)
+    assert len(gpu_keep) == len(want) == min(k, n)
+    assert np.all(np.diff(gpu_keep) > 0)
+    if np.array_equal(gpu_keep, want) or k <= 0 or k >= n:
+        assert np.array_equal(gpu_keep, want)
+        return 0
+    s = -score64 if largest else score64
+    srt = np.sort(s)
+    lo, hi = srt[k - 1], srt[k]
+    band = (s >= lo - rtol * abs(lo)) & (s <= hi + rtol * abs(hi))
+    diff = np.setxor1d(gpu_keep, want)
+    assert np.all(band[diff]), f"{len(diff)} tokens outside the tolerance band differ"
+    return int(len(diff))
+
+
+def rel_err(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return np.abs(a - b) / np.maximum(np.abs(b), 1e-300)
+
+
+class GpuFilterResult:
+    pass
+
+
+def gpu_filter(feat_bits, pos, metric, d_c, tau, n_centers, alpha=0.05):
+    feat = vb.bf16_tensor(feat_bits)
+    B, n, D = feat.shape
+    p = None if pos is None else torch.from_numpy(np.ascontiguousarray(pos, dtype=np.float32)).to(DEV)
+    label = torch.full((B, n), -5, dtype=torch.int32, device=DEV)
+    ncl = torch.full((B,), -5, dtype=torch.int32, device=DEV)
+    rho = torch.zeros((B, n), dtype=torch.float32, device=DEV)
+    d2 = torch.zeros((B, n), dtype=torch.float32, device=DEV)
+    par = torch.full((B, n), -5, dtype=torch.int32, device=DEV)
+    ws = vb.alloc_workspace(vb.OP_FILTER, B=B, Nv=n, D=D)
+    vb.vitcop_redundancy_filter(feat, p, label, ncl, ws, metric=metric, d_c=d_c, tau=tau, alpha=alpha,
+                                n_centers=n_centers, rho=rho, delta2=d2, parent=par)
+    status = vb.vitcop_poll_status(ws)
+    r = GpuFilterResult()
+    r.label, r.n_clusters = label.cpu().numpy(), ncl.cpu().numpy()
+    r.rho, r.delta2, r.parent = rho.cpu().numpy(), d2.cpu().numpy(), par.cpu().numpy()
+    r.status = status
+    return r
+
+
+def gpu_similarity_rows(feat_bits, metric, r0, r1):
+    feat = vb.bf16_tensor(feat_bits)
+    B, n, D = feat.shape
+    out = torch.full((B, r1 - r0, n), 9.0, dtype=torch.float32, device=DEV)
+    ws = vb.alloc_workspace(vb.OP_SIMILARITY, B=B, Nv=n, D=D)
+    vb.vitcop_similarity_rows(feat, metric, r0, r1, out, ws)
+    assert vb.vitcop_poll_status(ws) == vb.OK
+    return out.cpu().numpy()
+
+
+def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta2, g_parent, g_label, report=None):
+    """Three-level comparison of one sample of the filter against the oracle (see DESIGN notes).
+
+    1. continuous: rho, delta^2 within tolerance;
+    2. discrete vs the oracle: parents / centres / labels equal wherever no decision on the token's path
+       lies inside the tolerance band ("fragile" tokens are excluded and counted);
+    3. self-consistency, no band: the oracle's discrete steps re-run on the GPU's own fp32 rho / delta^2 /
+       parent must reproduce the GPU's parents (up to exact-tie fragility), centres and labels.
+    """
+    n = feat_bits.shape[0]
+    o = oracle.vic(feat_bits, pos, metric, d_c, tau, n_centers, tols=VIC_TOLS)
+    # ---- level 1
+    assert np.all(rel_err(g_rho, o["rho"]) <= RHO_RTOL), f"rho rel err {rel_err(g_rho, o['rho']).max():.3g}"
+    frag = o["fragile"].astype(bool)
+    same_parent = g_parent == o["parent"]
+    assert np.all(same_parent[~frag]), f"{(~same_parent & ~frag).sum()} robust parents differ"
+    fin = np.isfinite(o["delta2"]) & same_parent
+    assert np.all(np.isinf(g_delta2[same_parent & ~np.isfinite(o["delta2"])]))
+    err = np.abs(g_delta2[fin].astype(np.float64) - o["delta2"][fin])
+    assert np.all(err <= D2_ATOL + D2_RTOL * o["delta2"][fin]), f"delta2 err {err.max():.3g}"
+    # ---- level 3a: parents from the GPU's own rho (only exact-tie / near-tie in d2 or space can differ)
+    rho_g64 = g_rho.astype(np.float64)
+    d2sc, psc, fsc = oracle.vic_parents(o["d2"], pos, rho_g64, tau, tol_rho=0.0, tol_d2_abs=D2_ATOL,
+                                        tol_d2_rel=D2_RTOL, tol_sp=1e-6, want_fragile=True)
+    fsc = fsc.astype(bool)
+    assert np.all((g_parent == psc)[~fsc]), "parents inconsistent with the GPU's own densities"
+    # ---- level 3b: centres from the GPU's own (rho, delta2); gamma is compared with a 1e-6 relative guard
+    g_isc = (g_label == np.arange(n))
+    assert g_isc.sum() == min(n_centers, n)
+    d2_g64 = g_delta2.astype(np.float64)
+    isc_sc, gamma_sc, rank_sc = oracle.vic_centers(rho_g64, d2_g64, n_centers)
+    if not np.array_equal(g_isc, isc_sc.astype(bool)):
+        nc = min(n_centers, n)
+        cut_in, cut_out = gamma_sc[rank_sc[nc - 1]], gamma_sc[rank_sc[nc]]
+        diff = np.flatnonzero(g_isc != isc_sc.astype(bool))
+        near = np.abs(gamma_sc[diff] - cut_in) <= 1e-6 * abs(cut_in)
+        near |= np.abs(gamma_sc[diff] - cut_out) <= 1e-6 * abs(cut_out)
+        assert np.all(near), "centre set inconsistent with the GPU's own rho/delta2"
+    # ---- level 3c: labels from the GPU's own parents and centres (pure integer work + orphan fallback)
+    lab_sc = oracle.vic_labels(o["d2"], rho_g64, g_parent, g_isc.astype(np.uint8))
+    cs = np.flatnonzero(g_isc)
+    for i in np.flatnonzero(lab_sc != g_label):
+        # only tokens hanging below a surplus orphan may differ, and only if that orphan's nearest
+        # centre is a near-tie in d2
+        r = int(i)
+        while not g_isc[r] and g_parent[r] >= 0:
+            r = int(g_parent[r])
+        assert not g_isc[r] and g_parent[r] < 0, "labels inconsistent with the GPU's own parents/centres"
+        assert g_label[i] == g_label[r]
+        dd = o["d2"][r, cs]
+        assert abs(o["d2"][r, g_label[r]] - dd.min()) <= D2_ATOL + D2_RTOL * dd.min(), "orphan fallback inconsistent"
+    assert set(np.unique(g_label).tolist()) <= set(np.flatnonzero(g_isc).tolist())
+    # ---- level 2: against the oracle's own discrete results
+    o_isc = o["is_center"].astype(bool)
+    centres_equal = np.array_equal(o_isc, g_isc)
+    n_frag_label = n
+    if centres_equal:
+        # a token is label-robust when every token on its parent chain (up to its root) is parent-robust
+        robust = ~frag
+        chain_ok = robust.copy()
+        order = np.argsort(-o["rho"], kind="stable")
+        for i in order:                       # parents precede children in this order
+            p = o["parent"][i]
+            if not o_isc[i] and p >= 0:
+                chain_ok[i] = robust[i] and chain_ok[p]
+        cmp = chain_ok & ~((o["parent"] < 0) & ~o_isc)
+        assert np.array_equal(g_label[cmp], o["label"][cmp]), "robust labels differ from the oracle"
+        n_frag_label = int((~cmp).sum())
+    if report is not None:
+        report.append(dict(n=n, fragile_parent=int(frag.sum()), parent_mismatch=int((~same_parent).sum()),
+                           centres_equal=bool(centres_equal), label_uncompared=n_frag_label,
+                           label_mismatch=int((g_label != o["label"]).sum()),
+                           rho_err=float(rel_err(g_rho, o["rho"]).max())))
+    return o
