@@ -91,7 +91,8 @@ typedef struct {
     int   metric;      /* 0 cosine, 1 euclid */
     float d_c;         /* cutoff distance of Eq. 2 (> 0) */
     float tau;         /* spatial threshold of Eq. 3 on the coordinates in `pos`; < 0 disables the test */
-    float alpha;       /* centre ratio: n_centers = ceil(n * alpha) evaluated in double; used when n_centers <= 0 */
+    double alpha;      /* centre ratio: n_centers = ceil(n * alpha) evaluated in double (a float 0.05 would make
+                          200 * alpha exceed 10 and round up to 11); used when n_centers <= 0 */
     int   n_centers;   /* > 0 overrides alpha; clamped to n */
 } vitcop_filter_params;
 

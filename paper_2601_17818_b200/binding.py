@@ -38,7 +38,7 @@ class VitcopError(RuntimeError):
 
 
 class FilterParams(C.Structure):
-    _fields_ = [("metric", C.c_int), ("d_c", C.c_float), ("tau", C.c_float), ("alpha", C.c_float),
+    _fields_ = [("metric", C.c_int), ("d_c", C.c_float), ("tau", C.c_float), ("alpha", C.c_double),
                 ("n_centers", C.c_int)]
 
 

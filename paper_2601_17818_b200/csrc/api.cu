@@ -212,7 +212,7 @@ int vitcop_redundancy_filter(const void* feat, const float* pos, int B, int n, i
         return VITCOP_ERR_WORKSPACE;
     int nc = p->n_centers;
     if (nc <= 0) {
-        const double v = std::ceil((double)n * (double)p->alpha);
+        const double v = std::ceil((double)n * p->alpha);
         nc = v < 0 ? 0 : (v > n ? n : (int)v);
     }
     if (nc > n) nc = n;

@@ -32,7 +32,8 @@ constexpr int BK = 64;             // k-block: 64 bf16 = 128 bytes = one 128B-sw
 constexpr int UMMA_K = 16;
 constexpr int kGemmThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 constexpr int kEpiThreads = 128;
-constexpr uint32_t kSpinLimit = 1u << 22;   // bounded waits: give up, flag VITCOP_ERR_TIMEOUT and leave
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s give up, flag VITCOP_ERR_TIMEOUT and leave
+constexpr unsigned long long kDrainLimitNs = 20000000ull;    // bounded waits for this CTA's own copies / MMAs after giving up
 
 enum { MODE_RHO = 0, MODE_DELTA = 1, MODE_SIM = 2 };
 
@@ -79,14 +80,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return done != 0;
 }
-// Bounded wait.  Returns false (after raising `abort_flag`) when the limit is hit or another role gave up.
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false (after raising `abort_flag`) when the time limit is hit or another role gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u && *abort_flag) return false;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) break;
+        }
     }
     *abort_flag = 1;
     return false;
+}
+// Bounded wait without side effects, used while leaving after a timeout.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const unsigned long long t0 = global_ns();
+    while (!mbar_try_wait(bar, parity))
+        if (global_ns() - t0 > kDrainLimitNs) break;
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
@@ -138,6 +155,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int u = 0; u < 32; ++u) v[u] = __uint_as_float(r[u]);
 }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ORs a predicate: every thread gets the same answer.
+__device__ __forceinline__ bool epi_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) wide,
 // laid out by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
@@ -306,12 +336,13 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t* gen = smem_raw + (tiles - raw);
     float* colbase = reinterpret_cast<float*>(gen + S::kTileBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kColBytes);
-    // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]
+    // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], drain
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * S::kStages;
     const uint32_t bar_tfull = bar_empty + 8 * S::kStages;
     const uint32_t bar_tempty = bar_tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + 4);
+    const uint32_t bar_drain = bar_tempty + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + 5);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -326,6 +357,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(bar_tfull + 8 * a, 1);
             mbar_init(bar_tempty + 8 * a, kEpiThreads);
         }
+        mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
@@ -347,6 +379,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0, issued_parity = 0;        // per stage: a load was issued / parity of its phase
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
                 const int b = (int)(t / tiles_per_b);
@@ -359,8 +392,15 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
                     tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
                     tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
+                    issued |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
                 }
+            }
+            if (!ok) {
+                // leaving early: give the copies still in flight into this CTA's shared memory time to land
+                for (int s = 0; s < S::kStages; ++s)
+                    if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
             }
         }
     } else if (warp == 1) {
@@ -391,6 +431,11 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!ok) break;
                 tc_commit(bar_tfull + 8 * acc);            // accumulator complete
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (!ok) {
+                // leaving early: let the MMAs already issued finish before TMEM is released
+                tc_commit(bar_drain);
+                mbar_drain(bar_drain, 0);
             }
         }
     } else {
@@ -430,8 +475,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 epi_row_end<MODE>(g, rs, b, tj, row_valid);
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
-            epi_bar_sync();                                // column arrays are rewritten for the next tile
-            if (!ok) break;
+            // column arrays are rewritten for the next tile; all four warps leave together or not at all
+            if (epi_bar_or(!ok)) break;
         }
     }
 

@@ -13,9 +13,22 @@ from paper_2601_17818_b200 import workloads as W
 KNORM_RTOL = 1e-5        # K-norm: |gpu - oracle| <= 1e-5 * oracle
 SIM_ATOL = 1e-5          # cosine similarity in [-1, 1]: absolute 1e-5
 GRAM_RTOL = 1e-5         # raw Gram (euclid): |gpu - oracle| <= 1e-5 * sqrt(g_ii * g_jj)
-RHO_RTOL = 1e-5          # density
-D2_ATOL, D2_RTOL = 2e-5, 1e-5   # delta^2 (2 - 2s cancels for near-duplicates, hence the absolute part)
-VIC_TOLS = dict(tol_rho=RHO_RTOL, tol_d2_abs=D2_ATOL, tol_d2_rel=D2_RTOL, tol_sp=1e-6)
+D2_RTOL = 1e-5           # relative part of the delta^2 tolerance
+
+
+def vic_tolerances(metric, d_c, feat_bits):
+    """Tolerances of the quantities derived from the similarity, by propagating the similarity tolerance.
+
+    cosine:  d^2 = 2 - 2 s, so |err(d^2)| <= 2 * SIM_ATOL (absolute: the subtraction cancels for near-duplicates);
+    euclid:  d^2 = g_ii + g_jj - 2 g_ij, so |err(d^2)| <= 2 * GRAM_RTOL * max_i g_ii.
+    Each term exp(-d^2 / d_c^2) of Eq. 2 then moves by at most err(d^2) / d_c^2 relative, and so does rho
+    (a sum of positive terms)."""
+    if metric == 0:
+        d2_atol = 2.0 * SIM_ATOL
+    else:
+        x = W.bf16_bits_to_f32(feat_bits).astype(np.float64)
+        d2_atol = 2.0 * GRAM_RTOL * float((x * x).sum(-1).max())
+    return dict(d2_atol=d2_atol, d2_rtol=D2_RTOL, rho_rtol=d2_atol / (d_c * d_c))
 
 DEV = "cuda"
 
@@ -127,7 +140,10 @@ def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta
        parent must reproduce the GPU's parents (up to exact-tie fragility), centres and labels.
     """
     n = feat_bits.shape[0]
-    o = oracle.vic(feat_bits, pos, metric, d_c, tau, n_centers, tols=VIC_TOLS)
+    tol = vic_tolerances(metric, d_c, feat_bits)
+    RHO_RTOL, D2_ATOL = tol["rho_rtol"], tol["d2_atol"]
+    o = oracle.vic(feat_bits, pos, metric, d_c, tau, n_centers,
+                   tols=dict(tol_rho=RHO_RTOL, tol_d2_abs=D2_ATOL, tol_d2_rel=D2_RTOL, tol_sp=1e-6))
     # ---- level 1
     assert np.all(rel_err(g_rho, o["rho"]) <= RHO_RTOL), f"rho rel err {rel_err(g_rho, o['rho']).max():.3g}"
     frag = o["fragile"].astype(bool)
