@@ -2,19 +2,22 @@
 """Benchmark of the ViTCoP pruning operator chain on B200.
 
 One "step" = one pass of the whole hot path over one batch of the LLaVA-1.5-shaped batch-16 workload
-("c1"): redundancy filter (VIC clustering of the vision features) followed by the fused pruning step
-(K-norm -> cluster-quota selection -> compaction of hidden states, K and V).
+("c1"): redundancy filter (VIC clustering of the vision features, Algorithm 2) followed by the fused
+pruning step (K-norm, Eq. 4 -> cluster-quota selection, Eq. 5 -> compaction of hidden states, K and V).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c1]
 
 Prints ONE JSON line.  `value` is visual tokens pruned per second with the inputs resident in HBM
 (CUDA-event time per step, L2 flushed between steps); `e2e` is the same metric through the public API
-with pinned HOST buffers, host<->device copies inside the timed region.  `--impl reference` times the
-CPU oracle (test infrastructure) on the host cores instead.
+with pinned HOST buffers, host<->device copies inside the timed region; `roofline` describes the kernel
+that takes the largest share of the step, timed by CUDA events the library records around each of its
+kernels; `cpu_baseline` is the CPU oracle timed on the host cores.  `--impl reference` times that oracle
+(test infrastructure) instead of the CUDA path.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -30,7 +33,12 @@ from paper_2601_17818_b200 import workloads as W  # noqa: E402
 
 METRIC = "visual_tokens_pruned_per_s"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 8   # row_stats, gram(rho), rho_reduce, gram(delta), vic_finalize, knorm, select, compact
+
+# DRAM bytes (read + write) per launch from the committed ncu captures under profiles/: kernel name ->
+# (bytes per launch on the bench workload, sha1 of the kernel's source file when the counters were taken).
+# A kernel whose source changed since reports traffic null.
+NCU_TRAFFIC = {
+}
 
 
 def measured_peaks():
@@ -41,6 +49,19 @@ def measured_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
                     bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def source_sha(name: str) -> str:
+    with open(os.path.join(ROOT, "paper_2601_17818_b200", "csrc", name), "rb") as fh:
+        return hashlib.sha1(fh.read()).hexdigest()[:12]
+
+
+def config_of(w, **extra):
+    c = {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
+         "budget": w.budgets[0], "n_centers": w.n_centers, "d_c": w.d_c, "tau": w.tau,
+         "mode": "redundancy filter (cosine) + fused prune step in cluster-quota mode"}
+    c.update(extra)
+    return c
 
 
 # ------------------------------------------------------------------------------------------------ oracle legs
@@ -58,37 +79,55 @@ def oracle_step(w, feat, pos, K, V, hidden, budget):
     return pruned
 
 
-def time_oracle(w, steps, warmup, sample_B):
-    import oracle
-    feat, pos = W.make_features(w, B=sample_B), W.make_positions(w)[:sample_B]
-    K, V = W.make_kv(w, 0, w.Nv, B=sample_B)
-    hidden = W.make_hidden(w, B=sample_B)
-    oracle.build()
-    for _ in range(warmup):
-        oracle_step(w, feat, pos, K, V, hidden, w.budgets[0])
-    t0 = time.perf_counter()
-    pruned = 0
-    for _ in range(steps):
-        pruned += oracle_step(w, feat, pos, K, V, hidden, w.budgets[0])
-    dt = time.perf_counter() - t0
-    return pruned / dt, dt / steps, oracle.num_threads()
+class OracleBench:
+    """The CPU oracle on a bounded sample (the first `sample_B` sequences) of the workload."""
+
+    def __init__(self, w, sample_B):
+        import oracle
+        self.w, self.sample_B = w, sample_B
+        self.feat, self.pos = W.make_features(w, B=sample_B), W.make_positions(w)[:sample_B]
+        self.K, self.V = W.make_kv(w, 0, w.Nv, B=sample_B)
+        self.hidden = W.make_hidden(w, B=sample_B)
+        oracle.build()
+        self.cores = oracle.num_threads()
+
+    def step(self):
+        return oracle_step(self.w, self.feat, self.pos, self.K, self.V, self.hidden, self.w.budgets[0])
+
+    def run(self, steps, warmup):
+        for _ in range(warmup):
+            self.step()
+        t0 = time.perf_counter()
+        pruned = sum(self.step() for _ in range(steps))
+        dt = time.perf_counter() - t0
+        return pruned / dt, dt / steps
+
+    def run_for(self, seconds, warmup=1):
+        for _ in range(warmup):
+            self.step()
+        t0 = time.perf_counter()
+        pruned, steps = 0, 0
+        while steps < 3 or time.perf_counter() - t0 < seconds:
+            pruned += self.step()
+            steps += 1
+        dt = time.perf_counter() - t0
+        return pruned / dt, dt, steps
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     w = W.workload(args.workload)
     sample_B = min(w.B, 4)
-    value, sec_per_step, cores = time_oracle(w, args.steps, args.warmup, sample_B)
-    sample = f"{sample_B} of {w.B} samples of workload {w.name} per step (fp64 CPU oracle, whole hot path)"
+    ob = OracleBench(w, sample_B)
+    value, sec_per_step = ob.run(args.steps, args.warmup)
+    sample = (f"each step = the first {sample_B} of {w.B} sequences of workload {w.name}, whole hot path "
+              f"(fp64 CPU oracle, OpenMP over rows)")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
-                   "budget": w.budgets[0], "n_centers": w.n_centers},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_of(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": ob.cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -183,6 +222,44 @@ class Step:
         self.prune()
 
 
+def kernel_rooflines(w, nk_total, per_kernel, peaks):
+    """Roofline entry of every kernel that has one: algorithmic bytes or flops per launch / measured duration.
+
+    knorm:   reads the visual span of K once (B*H*Nv*d bf16) and writes B*Nv fp32 scores            -> HBM
+    compact: reads and writes every surviving row of hidden, K and V once, plus the index arrays    -> HBM
+    gram:    one sweep over the symmetric half of the Gram matrix incl. the diagonal, 2*D flop per pair,
+             B*n*(n+1)/2 pairs                                                                         -> tensor cores
+    The remaining kernels (row statistics, rho reduction, centres/labels, selection) move kilobytes and are
+    latency-bound; they are reported in microseconds only.
+    """
+    rows_out = w.B * w.T + nk_total
+    algo = {
+        "knorm_kernel": ("hbm", w.B * w.H * w.Nv * w.d * 2 + w.B * w.Nv * 4),
+        "compact_kernel": ("hbm", 2 * rows_out * (w.Dh + 2 * w.H * w.d) * 2 + rows_out * 4 + w.B * 12 + nk_total * 4),
+        "gram_tc_kernel<rho>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
+        "gram_tc_kernel<delta>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
+    }
+    src = {"knorm_kernel": "knorm.cu", "compact_kernel": "compact.cu", "gram_tc_kernel<rho>": "filter.cu",
+           "gram_tc_kernel<delta>": "filter.cu"}
+    out = {}
+    for name, (launches, ms) in per_kernel.items():
+        us = ms * 1e3 / max(launches, 1)
+        e = {"launches": launches, "us_per_launch": us}
+        if name in algo and us > 0:
+            bound, units = algo[name]
+            if bound == "hbm":
+                ach, peak, unit = units / (us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
+            else:
+                ach, peak, unit = units / (us * 1e-6) / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+            traffic = None
+            if name in NCU_TRAFFIC and NCU_TRAFFIC[name][1] == source_sha(src[name]):
+                traffic = NCU_TRAFFIC[name][0]
+            e.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=traffic,
+                     algorithmic_units_per_launch=units)
+        out[name] = e
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -235,22 +312,46 @@ def run_ours(args):
         barrier()
         return np.array([a.elapsed_time(b) for a, b in evs], dtype=np.float64)
 
+    def max_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
     # whole step, device resident ------------------------------------------------------------------------
     sampler = ClockSampler(local)
     sampler.start()
     t_step = timed(st.run, args.steps, args.warmup)
     clocks = sampler.stop()
     n_keep = st.nkeep.cpu().numpy()
+    nk_total = int(n_keep.sum())
     pruned_per_step = int((w.Nv - n_keep).sum())
-    total_ms = float(t_step.sum())
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(t_step.sum()))
     value = world * pruned_per_step * args.steps / (total_ms * 1e-3)
 
-    # per-stage times (same protocol) ------------------------------------------------------------------
-    stage = {}
+    # per-kernel device times: the library brackets each of its kernels with CUDA events on the stream ----
+    n_kt = max(10, min(args.steps, 50))
+    for _ in range(3):
+        flush.zero_()
+        st.run()
+    torch.cuda.synchronize()
+    vb.vitcop_kernel_timing_begin()
+    for _ in range(n_kt):
+        flush.zero_()
+        st.run()
+    per_kernel = vb.vitcop_kernel_timing_end()
+    kernels = kernel_rooflines(w, nk_total, per_kernel, peaks)
+    launches_per_step = sum(v[0] for v in per_kernel.values()) // n_kt
+    dom = max(per_kernel, key=lambda k: per_kernel[k][1])
+    roofline = {"kernel": dom}
+    roofline.update({k: kernels[dom].get(k) for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")})
+    roofline.update(peak_source=peaks["source"] + (" burst" if kernels[dom].get("bound") == "tensor" else " copy"),
+                    us_per_launch=kernels[dom]["us_per_launch"],
+                    algorithmic_units_per_launch=kernels[dom].get("algorithmic_units_per_launch"),
+                    share_of_step=per_kernel[dom][1] / sum(v[1] for v in per_kernel.values()))
+
+    # per-API-call times (same protocol as the step) -----------------------------------------------------------
     score = torch.empty((w.B, w.Nv), dtype=torch.float32, device=dev)
     kidx = torch.empty((w.B, w.Nv), dtype=torch.int32, device=dev)
     ws_sel = vb.alloc_workspace(vb.OP_SELECT, device=dev, B=w.B, Nv=w.Nv)
@@ -262,27 +363,10 @@ def run_ours(args):
                                                 st.Ko, st.Vo, st.olen, kept_pos=st.kpos),
         "prune_step": st.prune,
     }
-    n_stage = max(10, min(args.steps, 50))
+    stage = {}
     for name, fn in stage_fns.items():
-        t = timed(fn, n_stage, 3)
+        t = timed(fn, n_kt, 3)
         stage[name] = {"us_median": float(np.median(t) * 1e3), "us_min": float(t.min() * 1e3)}
-    nk_total = int(st.nkeep.cpu().numpy().sum())
-    knorm_bytes = w.B * w.H * w.Nv * w.d * 2 + w.B * w.Nv * 4
-    rows_out = w.B * w.T + nk_total
-    compact_bytes = 2 * rows_out * (w.Dh + 2 * w.H * w.d) * 2
-    gram_flop = w.B * w.Nv * (w.Nv + 1) * w.D            # algorithmic: symmetric half incl. diagonal
-    stage["knorm"].update(bytes=knorm_bytes, gbs=knorm_bytes / (stage["knorm"]["us_median"] * 1e-6) / 1e9)
-    stage["compact"].update(bytes=compact_bytes, gbs=compact_bytes / (stage["compact"]["us_median"] * 1e-6) / 1e9)
-    stage["filter"].update(algorithmic_flop=gram_flop,
-                           tflops=gram_flop / (stage["filter"]["us_median"] * 1e-6) / 1e12)
-    for k in ("knorm", "compact"):
-        stage[k]["frac_of_measured_hbm"] = stage[k]["gbs"] / peaks["hbm_gbs"]
-    # the dominant single kernel of the step
-    single = {"knorm": stage["knorm"]["us_median"], "compact": stage["compact"]["us_median"]}
-    dom = max(single, key=single.get)
-    roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": stage[dom]["gbs"], "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": stage[dom]["gbs"] / peaks["hbm_gbs"], "traffic": None,
-                "peak_source": peaks["source"], "algorithmic_bytes_per_launch": stage[dom]["bytes"]}
 
     # end to end through the public API with host buffers ----------------------------------------------------
     out_host = {"ho": torch.empty(st.ho.shape, dtype=st.ho.dtype).pin_memory(),
@@ -302,36 +386,32 @@ def run_ours(args):
 
     n_e2e = max(5, min(args.steps, 20))
     t_e2e = timed(e2e_step, n_e2e, 3)
-    e2e_ms = float(t_e2e.sum())
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(float(t_e2e.sum()))
     h2d = sum(int(v.numel() * v.element_size()) for v in host.values())
     d2h = sum(int(v.numel() * v.element_size()) for v in out_host.values())
     e2e = {"value": world * pruned_per_step * n_e2e / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / n_e2e}
 
-    # CPU oracle beside it (rank 0, N = 1 only; bounded sample) ------------------------------------------------
+    # CPU oracle beside it (rank 0, N = 1 only; bounded sample of about 10 s) ---------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_B = min(w.B, 4)
-        v, sec, cores = time_oracle(w, 3, 1, sample_B)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{sample_B} of {w.B} samples of workload {w.name}, 3 timed passes of the whole hot path "
-                         f"({sec:.2f} s each)"}
+        ob = OracleBench(w, sample_B)
+        v, secs, passes = ob.run_for(args.cpu_seconds)
+        cpu = {"value": v, "unit": UNIT, "cores": ob.cores, "kind": "oracle",
+               "sample": f"the first {sample_B} of {w.B} sequences of workload {w.name}, whole hot path, "
+                         f"{passes} passes in {secs:.1f} s"}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, fp32 arithmetic", "data": "synthetic",
-            "config": {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
-                       "budget": st.budget, "n_centers": w.n_centers, "mode": "filter + quota prune step",
-                       "tokens_pruned_per_step": pruned_per_step, "tokens_kept_per_step": nk_total,
-                       "l2": "flushed (512 MiB memset) before every timed step", "sharding": "replicas only"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu, "stages": stage,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_of(w, accumulate="f32", tokens_pruned_per_step=pruned_per_step,
+                                tokens_kept_per_step=nk_total,
+                                l2="flushed (512 MiB memset) before every timed step", sharding="replicas only"),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels, "stages": stage,
             "us_per_step_median": float(np.median(t_step) * 1e3),
         }
         print(json.dumps(line))
@@ -347,6 +427,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="length of the CPU-oracle timing leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

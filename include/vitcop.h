@@ -69,6 +69,23 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
  * workspace resets the word when it starts, so poll after the call of interest. */
 int vitcop_poll_status(const void* workspace, void* stream, int* device_status);
 
+/* ---------------------------------------------------------------- diagnostic: per-kernel device times
+ * The paper has no counterpart; this exists so that a benchmark can attribute the time of a multi-kernel
+ * call to its kernels.  Between vitcop_kernel_timing_begin and vitcop_kernel_timing_end every kernel the
+ * library launches (process-wide) is bracketed by two CUDA events on its stream, and kernels of one call
+ * no longer overlap (programmatic dependent launch is switched off), so a call runs slower than normal.
+ * vitcop_kernel_timing_end waits for the recorded events, sums launches and milliseconds per kernel name
+ * into out[0 .. *count) (host memory, at most `capacity` distinct names) and switches timing off.
+ * Not for use during stream capture.  Errors: INVALID_ARG, CUDA. */
+typedef struct {
+    char  name[48];     /* kernel name, NUL-terminated */
+    int   launches;
+    float total_ms;
+} vitcop_kernel_time;
+
+int vitcop_kernel_timing_begin(void);
+int vitcop_kernel_timing_end(vitcop_kernel_time* out, int capacity, int* count);
+
 /* ---------------------------------------------------------------- redundancy filter (VIC)
  * Visual Information Clustering, Algorithm 2 of the paper (Section "Visual Semantic Guidance",
  * Eq. 2 and Eq. 3): pairwise feature distance d_ij, local density

@@ -24,7 +24,7 @@ MAX_VISUAL_TOKENS = 16384
 EXPORTS = [
     "vitcop_status_string", "vitcop_last_cuda_error", "vitcop_workspace_bytes", "vitcop_poll_status",
     "vitcop_redundancy_filter", "vitcop_similarity_rows", "vitcop_knorm_score", "vitcop_select",
-    "vitcop_compact_kv", "vitcop_prune_step",
+    "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
 ]
 
 
@@ -40,6 +40,10 @@ class VitcopError(RuntimeError):
 class FilterParams(C.Structure):
     _fields_ = [("metric", C.c_int), ("d_c", C.c_float), ("tau", C.c_float), ("alpha", C.c_double),
                 ("n_centers", C.c_int)]
+
+
+class KernelTime(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_int), ("total_ms", C.c_float)]
 
 
 class SelectParams(C.Structure):
@@ -71,6 +75,8 @@ def lib() -> C.CDLL:
                                         vp, vp, vp, i32, vp, vp, vp]
         L.vitcop_prune_step.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, vp, i32, i32, vp, i32,
                                         vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.vitcop_kernel_timing_begin.argtypes = []
+        L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
             getattr(L, name)
         _lib = L
@@ -202,6 +208,18 @@ def vitcop_similarity_rows(feat: torch.Tensor, metric: int, row_begin: int, row_
                                       _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "vitcop_similarity_rows")
     return out
+
+
+def vitcop_kernel_timing_begin() -> None:
+    _check(lib().vitcop_kernel_timing_begin(), "vitcop_kernel_timing_begin")
+
+
+def vitcop_kernel_timing_end(capacity: int = 32) -> dict:
+    """{kernel name: (launches, total milliseconds)} of the kernels launched since ``vitcop_kernel_timing_begin``."""
+    buf = (KernelTime * capacity)()
+    n = C.c_int(0)
+    _check(lib().vitcop_kernel_timing_end(buf, capacity, C.byref(n)), "vitcop_kernel_timing_end")
+    return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(n.value)}
 
 
 # ----------------------------------------------------------------------------------------------

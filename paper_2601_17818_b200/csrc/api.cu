@@ -1,6 +1,10 @@
 // Public C ABI of libvitcop: argument validation, workspace carving and dispatch to the launchers.
+#include <atomic>
 #include <cmath>
 #include <cstdint>
+#include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "internal.cuh"
 
@@ -12,6 +16,40 @@ int record_cuda(cudaError_t e) {
     if (e == cudaSuccess) return VITCOP_OK;
     g_last_cuda_error = static_cast<int>(e);
     return VITCOP_ERR_CUDA;
+}
+
+// ---- diagnostic kernel timing ------------------------------------------------------------------------
+namespace {
+struct TimedLaunch {
+    const char* name;
+    cudaEvent_t start, stop;
+    bool complete;
+};
+std::atomic<bool> g_timing_on{false};
+std::mutex g_timing_mutex;
+std::vector<TimedLaunch> g_timed;
+}  // namespace
+
+bool kernel_timing_on() { return g_timing_on.load(std::memory_order_relaxed); }
+
+KernelTimeScope::KernelTimeScope(const char* name, cudaStream_t stream) : slot_(-1), stream_(stream) {
+    if (!kernel_timing_on()) return;
+    TimedLaunch t{name, nullptr, nullptr, false};
+    if (cudaEventCreate(&t.start) != cudaSuccess) return;
+    if (cudaEventCreate(&t.stop) != cudaSuccess) { cudaEventDestroy(t.start); return; }
+    cudaEventRecord(t.start, stream);
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    slot_ = (int)g_timed.size();
+    g_timed.push_back(t);
+}
+
+KernelTimeScope::~KernelTimeScope() {
+    if (slot_ < 0) return;
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    if (slot_ < (int)g_timed.size()) {
+        cudaEventRecord(g_timed[slot_].stop, stream_);
+        g_timed[slot_].complete = true;
+    }
 }
 
 namespace {
@@ -72,6 +110,43 @@ const char* vitcop_status_string(int status) {
 }
 
 int vitcop_last_cuda_error(void) { return g_last_cuda_error; }
+
+int vitcop_kernel_timing_begin(void) {
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    for (auto& t : g_timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+    g_timed.clear();
+    g_timing_on.store(true);
+    return VITCOP_OK;
+}
+
+int vitcop_kernel_timing_end(vitcop_kernel_time* out, int capacity, int* count) {
+    if (!count || capacity < 0 || (capacity > 0 && !out)) return VITCOP_ERR_INVALID_ARG;
+    g_timing_on.store(false);
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    int n = 0, rc = VITCOP_OK;
+    for (auto& t : g_timed) {
+        float ms = 0.f;
+        if (t.complete && rc == VITCOP_OK) {
+            rc = record_cuda(cudaEventSynchronize(t.stop));
+            if (rc == VITCOP_OK) rc = record_cuda(cudaEventElapsedTime(&ms, t.start, t.stop));
+            if (rc == VITCOP_OK) {
+                int k = 0;
+                while (k < n && std::strncmp(out[k].name, t.name, sizeof(out[k].name) - 1) != 0) ++k;
+                if (k == n && n < capacity) {
+                    std::memset(&out[n], 0, sizeof(out[n]));
+                    std::strncpy(out[n].name, t.name, sizeof(out[n].name) - 1);
+                    ++n;
+                }
+                if (k < n) { out[k].launches += 1; out[k].total_ms += ms; }
+            }
+        }
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    g_timed.clear();
+    *count = n;
+    return rc;
+}
 
 int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, int Dh, size_t* bytes) {
     (void)H; (void)N; (void)d; (void)Dh;

@@ -135,7 +135,8 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
+    KernelTimeScope timed("compact_kernel", stream);
     return record_cuda(cudaLaunchKernelEx(
         &cfg, compact_kernel, static_cast<const uint4*>(hidden), static_cast<const uint4*>(K),
         static_cast<const uint4*>(V), H, N, d / 8, Dh / 8, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,

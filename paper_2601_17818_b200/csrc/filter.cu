@@ -855,7 +855,8 @@ int launch_gram_tc(const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs&
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
+    KernelTimeScope timed(MODE == MODE_RHO ? "gram_tc_kernel<rho>" : MODE == MODE_DELTA ? "gram_tc_kernel<delta>" : "gram_tc_kernel<sim>", stream);
     return record_cuda(cudaLaunchKernelEx(&cfg, gram_tc_kernel<BN, MODE>, ma, mb, g));
 }
 
@@ -867,6 +868,7 @@ int launch_gram(const void* feat, GemmArgs g, cudaStream_t stream, bool pdl, int
         g.TJ = (g.n + 127) / 128;
         if (tj_used) *tj_used = g.TJ;
         dim3 grid(g.TJ, g.TI, g.B);
+        KernelTimeScope timed("gram_simt_kernel", stream);
         gram_simt_kernel<MODE><<<grid, kEpiThreads, 0, stream>>>(static_cast<const uint16_t*>(feat), g);
         return record_cuda(cudaGetLastError());
     }
@@ -922,9 +924,13 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     float* part = reinterpret_cast<float*>(ws + l.off_part);
 
     const int rows = B * n;
-    row_stats_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(feat), rows, D / 8, p.metric, w, a,
-                                                         best);
-    int rc = record_cuda(cudaGetLastError());
+    int rc;
+    {
+        KernelTimeScope timed("row_stats_kernel", stream);
+        row_stats_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(feat), rows, D / 8, p.metric, w,
+                                                             a, best);
+        rc = record_cuda(cudaGetLastError());
+    }
     if (rc != VITCOP_OK) return rc;
 
     GemmArgs g = {};
@@ -946,7 +952,8 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = pdl_allowed(true) ? 1 : 0;
+        KernelTimeScope timed("rho_reduce_kernel", stream);
         rc = record_cuda(cudaLaunchKernelEx(&cfg, rho_reduce_kernel, (const float*)part, B, n, TJ, l.n_pad, rho,
                                             rho_user));
         if (rc != VITCOP_OK) return rc;
@@ -969,7 +976,8 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_allowed(true) ? 1 : 0;
+    KernelTimeScope timed("vic_finalize_kernel", stream);
     return record_cuda(cudaLaunchKernelEx(&cfg, vic_finalize_kernel, static_cast<const uint16_t*>(feat), n, D, nc,
                                           (const float*)rho, (const unsigned long long*)best, (const float*)w,
                                           (const float*)a, label, n_clusters, delta2_user, parent_user));
@@ -981,9 +989,13 @@ int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, in
     float* w = reinterpret_cast<float*>(ws + kStatusBytes);
     float* a = reinterpret_cast<float*>(ws + kStatusBytes + align_up((size_t)B * n * 4, 256));
     const int rows = B * n;
-    row_stats_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(feat), rows, D / 8, metric, w, a,
-                                                         nullptr);
-    int rc = record_cuda(cudaGetLastError());
+    int rc;
+    {
+        KernelTimeScope timed("row_stats_kernel", stream);
+        row_stats_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(feat), rows, D / 8, metric, w, a,
+                                                             nullptr);
+        rc = record_cuda(cudaGetLastError());
+    }
     if (rc != VITCOP_OK) return rc;
     GemmArgs g = {};
     g.B = B; g.n = n; g.D = D; g.row0 = row_begin; g.row_end = row_end; g.metric = metric;

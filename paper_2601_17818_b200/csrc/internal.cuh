@@ -16,6 +16,21 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Records the first failing CUDA runtime error of the calling thread.
 int record_cuda(cudaError_t e);
 
+// Diagnostic per-kernel timing (vitcop_kernel_timing_begin / _end).  While it is on, a KernelTimeScope
+// around a launch records one CUDA event before and one after the kernel on its stream, and launchers
+// drop the programmatic-dependent-launch attribute so that consecutive kernels do not overlap.
+bool kernel_timing_on();
+struct KernelTimeScope {
+    KernelTimeScope(const char* name, cudaStream_t stream);
+    ~KernelTimeScope();
+    KernelTimeScope(const KernelTimeScope&) = delete;
+    KernelTimeScope& operator=(const KernelTimeScope&) = delete;
+private:
+    int slot_;
+    cudaStream_t stream_;
+};
+inline bool pdl_allowed(bool requested) { return requested && !kernel_timing_on(); }
+
 // ---- launchers (enqueue on `stream`, return VITCOP_OK or VITCOP_ERR_CUDA) -------------------------
 int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
                  int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,

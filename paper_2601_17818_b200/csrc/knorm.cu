@@ -83,6 +83,7 @@ int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t s
     auto go = [&](auto kern, int lpr) {
         const int tok = kKnormThreads / lpr;
         dim3 grid((span + tok - 1) / tok, B);
+        KernelTimeScope timed("knorm_kernel", stream);
         kern<<<grid, kKnormThreads, 0, stream>>>(Kp, H, d8, sb, sh, sn, vis_start, vis_len, vis_len_uniform, score,
                                                   Nv_cap);
     };

@@ -274,7 +274,7 @@ int launch_select(const float* score, const int32_t* label, int B, const int32_t
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
     const int cap = Nv_cap > 0 ? Nv_cap : 1;
     if (mode == 0) {
         const size_t smem = (size_t)cap * sizeof(uint32_t);
@@ -284,6 +284,7 @@ int launch_select(const float* score, const int32_t* label, int B, const int32_t
             if (e != cudaSuccess) return record_cuda(e);
         }
         cfg.dynamicSmemBytes = smem;
+        KernelTimeScope timed("select_plain_kernel", stream);
         return record_cuda(cudaLaunchKernelEx(&cfg, select_plain_kernel, score, vis_len, vis_len_uniform, Nv_cap,
                                               largest, budget, keep_idx, keep_stride, n_keep, keep_mask));
     }
@@ -296,6 +297,7 @@ int launch_select(const float* score, const int32_t* label, int B, const int32_t
         if (e != cudaSuccess) return record_cuda(e);
     }
     cfg.dynamicSmemBytes = smem;
+    KernelTimeScope timed("select_quota_kernel", stream);
     return record_cuda(cudaLaunchKernelEx(&cfg, select_quota_kernel, score, label, vis_len, vis_len_uniform, Nv_cap,
                                           P, budget, keep_idx, keep_stride, n_keep, keep_mask, status_word));
 }
