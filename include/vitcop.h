@@ -215,6 +215,34 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V,
                       float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------- fused pruning step without a workspace
+ * The paper has no counterpart: this is vitcop_prune_step for callers that have no way to obtain device
+ * memory for a workspace at the point of the call -- code that runs where cudaMalloc is off limits (inside a
+ * serving loop that must not touch the allocator, a plugin that is handed tensors but no allocator, a
+ * latency-critical path where an allocation could stall on another stream's work).  Same arguments and
+ * results as vitcop_prune_step, minus `workspace`: the scratch (status word, scores, keep list, counts) is a
+ * buffer of VITCOP_STATIC_SCRATCH_BYTES built into the library image, which every GPU that loads the library
+ * holds until the process exits.  The call allocates and frees nothing.
+ *   - Limit: vitcop_workspace_bytes(VITCOP_OP_PRUNE_STEP, B, .., Nv_cap, ..) must not exceed
+ *     VITCOP_STATIC_SCRATCH_BYTES (roughly B * Nv_cap <= 520,000); larger problems return
+ *     VITCOP_ERR_UNSUPPORTED and nothing is launched.
+ *   - The first call on each device looks up the buffer's device address (with that device current).  Make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one buffer and it keeps what the last call left; each call resets the
+ *     status word it needs zeroed and overwrites the rest before reading it.  Two calls whose work overlaps on
+ *     the GPU (different streams, no ordering between them) race on the buffer: order them.
+ *   - The device status word cannot be polled here; a quota budget below the cluster count shows as
+ *     n_keep_out[b] == 0 and out_len[b] == text length. */
+#define VITCOP_STATIC_SCRATCH_BYTES (4u << 20)
+
+int vitcop_prune_step_static(const void* hidden, const void* K, const void* V,
+                             int B, int H, int N, int d, int Dh, const int32_t* seq_len,
+                             int vis_start, const int32_t* vis_len, int vis_len_uniform, int Nv_cap,
+                             const int32_t* label, int budget,
+                             void* hidden_out, void* K_out, void* V_out, int Ncap,
+                             int32_t* kept_pos, int32_t* out_len,
+                             float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ EXPORTS = [
     "vitcop_status_string", "vitcop_last_cuda_error", "vitcop_workspace_bytes", "vitcop_poll_status",
     "vitcop_redundancy_filter", "vitcop_similarity_rows", "vitcop_knorm_score", "vitcop_select",
     "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
+    "vitcop_prune_step_static",
 ]
 
 
@@ -75,6 +76,8 @@ def lib() -> C.CDLL:
                                         vp, vp, vp, i32, vp, vp, vp]
         L.vitcop_prune_step.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, vp, i32, i32, vp, i32,
                                         vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.vitcop_prune_step_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, vp, i32, i32, vp, i32,
+                                               vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.vitcop_kernel_timing_begin.argtypes = []
         L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
@@ -184,6 +187,27 @@ def vitcop_prune_step(hidden, K, V, vis_start: int, vis_len, Nv_cap: int, budget
                                  Ncap, _ptr(kept_pos), _ptr(out_len), _ptr(score_out), _ptr(keep_idx_out),
                                  _ptr(n_keep_out), _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "vitcop_prune_step")
+    return out_len
+
+
+def vitcop_prune_step_static(hidden, K, V, vis_start: int, vis_len, Nv_cap: int, budget: int, hidden_out, K_out,
+                             V_out, out_len, label=None, kept_pos=None, seq_len=None, score_out=None,
+                             keep_idx_out=None, n_keep_out=None):
+    """``vitcop_prune_step`` on the library's built-in scratch buffer: no workspace argument, nothing allocated.
+
+    For callers that cannot get device memory at the point of the call.  Raises ``VitcopError`` with
+    ``ERR_UNSUPPORTED`` when the problem needs more than the built-in 4 MiB.  Calls share that buffer, so
+    calls that could overlap on the GPU must be ordered by the caller.
+    """
+    B, H, N, d = K.shape
+    Ncap = K_out.shape[2] if K_out is not None else hidden_out.shape[1]
+    Dh = hidden.shape[2] if hidden is not None else 0
+    vp, vu = _vis(vis_len)
+    rc = lib().vitcop_prune_step_static(_ptr(hidden), _ptr(K), _ptr(V), B, H, N, d, Dh, _ptr(seq_len), vis_start, vp,
+                                        vu, int(Nv_cap), _ptr(label), int(budget), _ptr(hidden_out), _ptr(K_out),
+                                        _ptr(V_out), Ncap, _ptr(kept_pos), _ptr(out_len), _ptr(score_out),
+                                        _ptr(keep_idx_out), _ptr(n_keep_out), _stream())
+    _check(rc, "vitcop_prune_step_static")
     return out_len
 
 

@@ -94,6 +94,37 @@ int check_span(int N, int vis_start, const int32_t* vis_len, int vis_len_uniform
 
 using namespace vitcop;
 
+// ---- built-in scratch of vitcop_prune_step_static ------------------------------------------------------
+// Lives in every GPU that loads the library, from load to exit.  In host code the array's name is only a
+// stand-in for the symbol, not a device address: the address each device gives it is looked up once per
+// device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+constexpr size_t kStaticScratchBytes = VITCOP_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up on the first call per device).
+int static_scratch_address(void** out) {
+    int dev = -1;
+    int rc = record_cuda(cudaGetDevice(&dev));
+    if (rc != VITCOP_OK) return rc;
+    if (dev < 0 || dev >= kMaxDevices) return VITCOP_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        rc = record_cuda(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (rc != VITCOP_OK) return rc;
+        if (!p) return VITCOP_ERR_CUDA;
+        g_scratch_addr[dev] = p;
+    }
+    *out = g_scratch_addr[dev];
+    return VITCOP_OK;
+}
+}  // namespace
+
 extern "C" {
 
 const char* vitcop_status_string(int status) {
@@ -274,6 +305,21 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, i
     if (rc != VITCOP_OK) return rc;
     return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep, Nv_cap,
                           nkeep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, s, true);
+}
+
+int vitcop_prune_step_static(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                             const int32_t* seq_len, int vis_start, const int32_t* vis_len, int vis_len_uniform,
+                             int Nv_cap, const int32_t* label, int budget, void* hidden_out, void* K_out, void* V_out,
+                             int Ncap, int32_t* kept_pos, int32_t* out_len, float* score_out, int32_t* keep_idx_out,
+                             int32_t* n_keep_out, void* stream) {
+    if (B < 0 || Nv_cap < 0) return VITCOP_ERR_INVALID_ARG;
+    if (StepWs(B, Nv_cap).total > kStaticScratchBytes) return VITCOP_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != VITCOP_OK) return rc;
+    return vitcop_prune_step(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, Nv_cap, label,
+                             budget, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, score_out, keep_idx_out,
+                             n_keep_out, scratch, kStaticScratchBytes, stream);
 }
 
 int vitcop_redundancy_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params* p,
