@@ -1,0 +1,686 @@
+// Tensor-core sweep over the Gram matrix of the visual-token features (Algorithm 2, step 1) with the
+// per-pair work of Eq. 2 (density) or Eq. 3 (nearest denser neighbour) fused into the epilogue.
+//
+// The Gram matrix f_I . f_J^T is taken on the RAW bf16 features (bf16 x bf16 products are exact in fp32) by
+// tcgen05.mma with fp32 accumulators in tensor memory; the L2 normalisation enters as fp32 factors in the
+// epilogue.  Nothing of size n^2 is ever written: the density sweep and the delta sweep each recompute the
+// tiles they need.
+//
+// Symmetry: d_ij = d_ji, so the two sweeps visit only tiles that hold a pair i < j.  Such a pair serves its
+// row token i (a per-thread accumulation along the row) and its column token j (a reduction over the 128
+// rows of the tile, done with a shuffle butterfly inside each warp and a fixed-order combination of the
+// four warps that share a column range).
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: feature tiles [128 x 64] and [BN x 64] (128-byte swizzle) into a ring of stages
+//   warp 1      one thread issues tcgen05.mma (M = 128, N = BN, K = 16) into one of two TMEM accumulators
+//   warps 2-9   epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 (its rows) and one half of the columns
+// Every wait is bounded; on expiry the CTA raises an abort flag, all roles leave, TMEM is released and
+// VITCOP_ERR_TIMEOUT is written to the status word.
+#include <cuda.h>
+
+#include "gram.cuh"
+
+namespace vitcop {
+namespace {
+
+constexpr int BM = kGramBM;
+constexpr int BK = 64;             // k-block: 64 bf16 = 128 bytes = one 128B-swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kGemmThreads = 64 + kEpiThreads;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s give up and leave
+constexpr unsigned long long kDrainLimitNs = 20000000ull;    // bounded waits for this CTA's own copies / MMAs after giving up
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false (after raising `abort_flag`) when the time limit is hit or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// Bounded wait without side effects, used while leaving after a timeout.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const unsigned long long t0 = global_ns();
+    while (!mbar_try_wait(bar, parity))
+        if (global_ns() - t0 > kDrainLimitNs) break;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int u = 0; u < 32; ++u) v[u] = __uint_as_float(r[u]);
+}
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barrier over the epilogue threads that also ORs a predicate: every thread gets the same answer.
+__device__ __forceinline__ bool epi_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, 256, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+// 2^x for x <= 0 (results below the normal range flush to zero); relative error about 2^-22.
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) wide,
+// laid out by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);          // start address
+    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;        // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                               // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                               // swizzle mode: 128 bytes
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------
+// tile numbering
+// ------------------------------------------------------------------------------------------------
+struct KernelArgs {
+    GramArgs g;
+    GramTiling t;
+    long long total_tiles;
+};
+
+template <int BN, bool SYM>
+__device__ __forceinline__ void decode_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
+    b = (int)(t / k.t.tiles_per_b);
+    const int r = (int)(t - (long long)b * k.t.tiles_per_b);
+    if (!SYM) {
+        ti = r / k.t.TJ;
+        tj = r - ti * k.t.TJ;
+        return;
+    }
+    constexpr int R = BN / BM;
+    int q = (int)((sqrtf(8.f * (float)r / (float)R + 1.f) - 1.f) * 0.5f);
+    while (q > 0 && R * q * (q + 1) / 2 > r) --q;
+    while (R * (q + 1) * (q + 2) / 2 <= r) ++q;
+    tj = q;
+    ti = r - R * q * (q + 1) / 2;
+}
+
+// ------------------------------------------------------------------------------------------------
+// warp butterflies: lane L ends up with the reduction over the 32 lanes of element L of the array
+// ------------------------------------------------------------------------------------------------
+template <int HALF, bool MIN>
+__device__ __forceinline__ void butterfly_stage(float* v, bool up) {
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) {
+        const float keep = up ? v[k + HALF] : v[k];
+        const float send = up ? v[k] : v[k + HALF];
+        const float recv = __shfl_xor_sync(0xffffffffu, send, HALF);
+        v[k] = MIN ? fminf(keep, recv) : keep + recv;
+    }
+}
+template <bool MIN>
+__device__ __forceinline__ float warp_transpose_reduce(float (&v)[32], int lane) {
+    butterfly_stage<16, MIN>(v, (lane & 16) != 0);
+    butterfly_stage<8, MIN>(v, (lane & 8) != 0);
+    butterfly_stage<4, MIN>(v, (lane & 4) != 0);
+    butterfly_stage<2, MIN>(v, (lane & 2) != 0);
+    butterfly_stage<1, MIN>(v, (lane & 1) != 0);
+    return v[0];
+}
+
+// ------------------------------------------------------------------------------------------------
+// shared memory
+// ------------------------------------------------------------------------------------------------
+template <int BN>
+struct GemmSmem {
+    static constexpr int kStages = (BN == 128) ? 6 : 4;
+    static constexpr int kABytes = BM * BK * 2;
+    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kTileBytes = kStages * kStageBytes;
+    // per column of the tile: w, a, rho, x, y; reduction scratch: 4 x value, 4 x index; per row: value, index
+    static constexpr int kEpiBytes = (5 + 4 + 4) * BN * 4 + 2 * BM * 4;
+    static constexpr int kBarBytes = 256;
+    static constexpr int kTotal = 1024 /*alignment slack*/ + kTileBytes + kEpiBytes + kBarBytes;
+};
+
+constexpr float kInf = __builtin_huge_valf();
+
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
+template <int BN, int MODE, int METRIC, bool SPATIAL>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const KernelArgs k) {
+    using S = GemmSmem<BN>;
+    constexpr bool SYM = MODE != GRAM_SIM;
+    const GramArgs& g = k.g;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned for the 128B swizzle
+    uint8_t* gen = smem_raw + (tiles - raw);
+    float* colw = reinterpret_cast<float*>(gen + S::kTileBytes);
+    float* cola = colw + BN;
+    float* colrho = cola + BN;
+    float* colx = colrho + BN;
+    float* coly = colx + BN;
+    float* colred = coly + BN;                                     // [4][BN]
+    int* colidx = reinterpret_cast<int*>(colred + 4 * BN);         // [4][BN]
+    float* rowred = reinterpret_cast<float*>(colidx + 4 * BN);     // [BM]
+    int* rowidx = reinterpret_cast<int*>(rowred + BM);             // [BM]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
+    // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], drain
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * S::kStages;
+    const uint32_t bar_tfull = bar_empty + 8 * S::kStages;
+    const uint32_t bar_tempty = bar_tfull + 16;
+    const uint32_t bar_drain = bar_tempty + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + 5);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr uint32_t kTmemCols = 2 * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S::kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, kEpiThreads);
+        }
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // The kernels that follow on the stream may be scheduled from here on; they wait for this grid to
+    // complete before they touch anything it writes.
+    grid_dependency_launch_dependents();
+
+    const long long total_tiles = k.total_tiles;
+    const int KB = g.D / BK;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        // The features are an input of the whole call (never written by the kernel before this one), so
+        // the loads need not wait for the preceding grid.
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0, issued_parity = 0;        // per stage: a load was issued / parity of its phase
+            bool ok = true;
+            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+                int b, ti, tj;
+                decode_tile<BN, SYM>(k, t, b, ti, tj);
+                const int I0 = g.row0 + ti * BM, J0 = tj * BN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = tiles + stage * S::kStageBytes;
+                    mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
+                    tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
+                    tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
+                    issued |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // leaving early: give the copies still in flight into this CTA's shared memory time to land
+                for (int s = 0; s < S::kStages; ++s)
+                    if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            uint32_t stage = 0, phase = 0;
+            uint32_t acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = tiles + stage * S::kStageBytes;
+                    const uint64_t da = umma_desc_k128(sa), db = umma_desc_k128(sa + S::kABytes);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                        // advancing 16 elements (32 bytes) along K inside the swizzle row: +2 in address units
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk), idesc,
+                                    (kb > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * stage);      // frees the smem stage once these MMAs have read it
+                    if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(bar_tfull + 8 * acc);            // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (!ok) {
+                // leaving early: let the MMAs already issued finish before TMEM is released
+                tc_commit(bar_drain);
+                mbar_drain(bar_drain, 0);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        const int e = threadIdx.x - 64;                    // 0..255
+        const int quarter = warp & 3;                      // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                  // which half of the tile's columns this warp handles
+        const int rl = quarter * 32 + lane;                // tile-local row == TMEM lane
+        constexpr int kChunks = BN / 64;                   // 32-column chunks per warp
+        const int rows_out = g.row_end - g.row0;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+
+        grid_dependency_wait();                            // w, a, rho, best come from the preceding kernels
+
+        for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            int b, ti, tj;
+            decode_tile<BN, SYM>(k, t, b, ti, tj);
+            const int I0 = g.row0 + ti * BM, J0 = tj * BN;
+            const int i = I0 + rl;
+            const bool row_valid = SYM ? (i < g.n) : (i < g.row_end);
+            const size_t bo = (size_t)b * g.n;
+
+            // ---- per-column and per-row constants
+            if (e < BN) {
+                const int j = J0 + e;
+                const bool cv = j < g.n;
+                colw[e] = cv ? g.w[bo + j] : 0.f;
+                if (METRIC == 1) cola[e] = cv ? g.a[bo + j] : 0.f;
+                if (MODE == GRAM_DELTA) {
+                    colrho[e] = cv ? g.rho[bo + j] : 0.f;
+                    if (SPATIAL) {
+                        colx[e] = cv ? g.pos[2 * (bo + j)] : 0.f;
+                        coly[e] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
+                    }
+                }
+            }
+            const float w_i = row_valid ? g.w[bo + i] : 0.f;
+            const float a_i = METRIC == 1 ? (row_valid ? g.a[bo + i] : 0.f) : 1.f;
+            const float m2w_i = -2.f * w_i;
+            float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
+            if (MODE == GRAM_DELTA && row_valid) {
+                rho_i = g.rho[bo + i];
+                if (SPATIAL) { x_i = g.pos[2 * (bo + i)]; y_i = g.pos[2 * (bo + i) + 1]; }
+            }
+            // every pair of the tile has i < j < n: no masking needed
+            const bool full = SYM && (J0 >= I0 + BM) && (J0 + BN <= g.n);
+
+            epi_bar_sync();
+            if (ok) ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+
+            float racc = 0.f;                              // GRAM_RHO: row-side sum
+            float rbest = kInf;                            // GRAM_DELTA: row-side minimum and its tile-local column
+            int rbest_c = -1;
+            if (ok) {
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + half * (BN / 2);
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    float v[32];
+                    tmem_ld32(taddr + c * 32, v);
+                    if (c == kChunks - 1) {
+                        // this thread has read all it needs from the accumulator
+                        tc_fence_before();
+                        mbar_arrive(bar_tempty + 8 * acc);
+                    }
+                    const int cl0 = half * (BN / 2) + c * 32;          // tile-local first column of the chunk
+                    if (MODE == GRAM_SIM) {
+                        if (row_valid) {
+                            float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
+#pragma unroll
+                            for (int u = 0; u < 32; ++u) {
+                                const int j = J0 + cl0 + u;
+                                if (j < g.n) o[j] = METRIC == 0 ? (v[u] * w_i) * colw[cl0 + u] : v[u];
+                            }
+                        }
+                    } else if (MODE == GRAM_RHO) {
+                        // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) {
+                            const float x = v[u] * colw[cl0 + u];
+                            const float base = METRIC == 0 ? 2.f : a_i + cola[cl0 + u];
+                            const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                            v[u] = ex2_approx(d2 * g.c2);
+                        }
+                        if (!full) {
+#pragma unroll
+                            for (int u = 0; u < 32; ++u) {
+                                const int j = J0 + cl0 + u;
+                                v[u] = (j > i && j < g.n && row_valid) ? v[u] : 0.f;
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) racc += v[u];
+                        const float cs = warp_transpose_reduce<false>(v, lane);
+                        colred[quarter * BN + cl0 + lane] = cs;
+                    } else {  // GRAM_DELTA, Eq. 3
+                        float kc[32];
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) {
+                            const float x = v[u] * colw[cl0 + u];
+                            const float base = METRIC == 0 ? 2.f : a_i + cola[cl0 + u];
+                            const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                            // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
+                            bool jd = colrho[cl0 + u] > rho_i;
+                            bool id = !jd;
+                            if (SPATIAL) {
+                                const float dx = colx[cl0 + u] - x_i, dy = coly[cl0 + u] - y_i;
+                                const bool near = fmaf(dx, dx, dy * dy) <= g.tau2;
+                                jd = jd && near;
+                                id = id && near;
+                            }
+                            if (!full) {
+                                const int j = J0 + cl0 + u;
+                                const bool pv = j > i && j < g.n && row_valid;
+                                jd = jd && pv;
+                                id = id && pv;
+                            }
+                            const float kr = jd ? d2 : kInf;
+                            kc[u] = id ? d2 : kInf;
+                            if (kr < rbest) { rbest = kr; rbest_c = cl0 + u; }
+                        }
+                        // column side: minimum over this warp's 32 rows, then the lowest row that attains it
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) v[u] = kc[u];
+                        const float cm = warp_transpose_reduce<true>(v, lane);
+                        uint32_t mine = 0;
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) {
+                            const float m = __shfl_sync(0xffffffffu, cm, u);
+                            const uint32_t bal = __ballot_sync(0xffffffffu, kc[u] == m && m < kInf);
+                            if (lane == u) mine = bal;
+                        }
+                        colred[quarter * BN + cl0 + lane] = cm;
+                        colidx[quarter * BN + cl0 + lane] = mine ? I0 + quarter * 32 + (__ffs(mine) - 1) : -1;
+                    }
+                }
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+
+            if (SYM) {
+                // ---- combine the two column halves of every row and the four row quarters of every column
+                if (half == 1) {
+                    rowred[rl] = MODE == GRAM_RHO ? racc : rbest;
+                    if (MODE == GRAM_DELTA) rowidx[rl] = rbest_c;
+                }
+                epi_bar_sync();
+                if (ok) {
+                    const int slot_base = b * k.t.slots();
+                    if (MODE == GRAM_RHO) {
+                        if (half == 0 && row_valid)
+                            g.part[((size_t)(slot_base + tj)) * k.t.n_pad + i] = racc + rowred[rl];
+                        if (e < BN && J0 + e < g.n)
+                            g.part[((size_t)(slot_base + k.t.TJ + ti)) * k.t.n_pad + J0 + e] =
+                                ((colred[e] + colred[BN + e]) + colred[2 * BN + e]) + colred[3 * BN + e];
+                    } else {
+                        if (half == 0 && row_valid) {
+                            const float other = rowred[rl];
+                            if (other < rbest) { rbest = other; rbest_c = rowidx[rl]; }   // tie: the lower column wins
+                            if (rbest_c >= 0) {
+                                const unsigned long long packed =
+                                    ((unsigned long long)__float_as_uint(rbest) << 32) |
+                                    (unsigned long long)(uint32_t)(J0 + rbest_c);
+                                atomicMin(g.best + bo + i, packed);
+                            }
+                        }
+                        if (e < BN && J0 + e < g.n) {
+                            float bk = kInf;
+                            int bi = -1;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {                                  // ascending rows: ties keep the lower row
+                                const float kk = colred[q * BN + e];
+                                if (kk < bk) { bk = kk; bi = colidx[q * BN + e]; }
+                            }
+                            if (bi >= 0) {
+                                const unsigned long long packed =
+                                    ((unsigned long long)__float_as_uint(bk) << 32) | (unsigned long long)(uint32_t)bi;
+                                atomicMin(g.best + bo + J0 + e, packed);
+                            }
+                        }
+                    }
+                }
+            }
+            // shared arrays are rewritten for the next tile; all epilogue warps leave together or not at all
+            if (epi_bar_or(!ok)) break;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && *abort_flag && g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 3-D view (D, n, B) of the bf16 feature tensor with a (64, box_rows, 1) box and the 128-byte swizzle.
+bool make_feat_map(CUtensorMap* map, const void* feat, int B, int n, int D, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)n, (cuuint64_t)B};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)n * D * 2};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(feat), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int num_sms() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    }
+    return sms;
+}
+
+template <int BN, int MODE, int METRIC, bool SPATIAL>
+int launch_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream, bool pdl) {
+    using S = GemmSmem<BN>;
+    static bool attr_done = false;
+    auto kern = gram_tc_kernel<BN, MODE, METRIC, SPATIAL>;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal);
+        if (e != cudaSuccess) return record_cuda(e);
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(k.total_tiles < num_sms() ? k.total_tiles : num_sms()));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = S::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
+    KernelTimeScope timed(MODE == GRAM_RHO ? "gram_tc_kernel<rho>"
+                                           : MODE == GRAM_DELTA ? "gram_tc_kernel<delta>" : "gram_tc_kernel<sim>",
+                          stream);
+    return record_cuda(cudaLaunchKernelEx(&cfg, kern, ma, mb, k));
+}
+
+template <int BN>
+int launch_bn(int mode, const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream,
+              bool pdl) {
+    const bool euclid = k.g.metric == 1;
+    const bool spatial = k.g.tau2 >= 0.f && k.g.pos != nullptr;
+    switch (mode) {
+        case GRAM_RHO:
+            return euclid ? launch_one<BN, GRAM_RHO, 1, false>(ma, mb, k, stream, pdl)
+                          : launch_one<BN, GRAM_RHO, 0, false>(ma, mb, k, stream, pdl);
+        case GRAM_DELTA:
+            if (spatial)
+                return euclid ? launch_one<BN, GRAM_DELTA, 1, true>(ma, mb, k, stream, pdl)
+                              : launch_one<BN, GRAM_DELTA, 0, true>(ma, mb, k, stream, pdl);
+            return euclid ? launch_one<BN, GRAM_DELTA, 1, false>(ma, mb, k, stream, pdl)
+                          : launch_one<BN, GRAM_DELTA, 0, false>(ma, mb, k, stream, pdl);
+        default:
+            return euclid ? launch_one<BN, GRAM_SIM, 1, false>(ma, mb, k, stream, pdl)
+                          : launch_one<BN, GRAM_SIM, 0, false>(ma, mb, k, stream, pdl);
+    }
+}
+
+}  // namespace
+
+int gram_pick_bn(int B, int n) {
+    const long long ti = (n + BM - 1) / BM;
+    const long long tiles128 = (long long)B * ti * (ti + 1) / 2;
+    return tiles128 >= 4LL * num_sms() ? 256 : 128;
+}
+
+int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream,
+                      bool pdl) {
+    KernelArgs k;
+    k.g = args;
+    k.t = tiling;
+    if (mode == GRAM_SIM) {
+        // plain rectangle: rows [row0, row_end) x all columns
+        const int rows = args.row_end - args.row0;
+        k.t.TI = (rows + BM - 1) / BM;
+        k.t.TJ = (args.n + tiling.BN - 1) / tiling.BN;
+        k.t.tiles_per_b = k.t.TI * k.t.TJ;
+    } else {
+        k.g.row0 = 0;
+        k.g.row_end = args.n;
+    }
+    k.total_tiles = (long long)args.B * k.t.tiles_per_b;
+    if (k.total_tiles <= 0) return VITCOP_OK;
+    CUtensorMap ma, mb;
+    if (!make_feat_map(&ma, feat, args.B, args.n, args.D, BM) ||
+        !make_feat_map(&mb, feat, args.B, args.n, args.D, tiling.BN))
+        return VITCOP_ERR_CUDA;
+    return tiling.BN == 256 ? launch_bn<256>(mode, ma, mb, k, stream, pdl)
+                            : launch_bn<128>(mode, ma, mb, k, stream, pdl);
+}
+
+}  // namespace vitcop

@@ -1,0 +1,61 @@
+// Interface between the tensor-core Gram sweep (gram.cu) and the rest of the redundancy filter (filter.cu).
+#pragma once
+
+#include "internal.cuh"
+
+namespace vitcop {
+
+constexpr int kGramBM = 128;   // rows of an output tile (UMMA M)
+
+enum GramMode { GRAM_RHO = 0, GRAM_DELTA = 1, GRAM_SIM = 2 };
+
+// Tiling of the symmetric sweeps (GRAM_RHO, GRAM_DELTA).  Only tiles that hold a pair (i, j) with i < j are
+// visited; a pair contributes to its row token i ("row side") and to its column token j ("column side").
+// Tiles are numbered column-tile major inside one sample: column tile tj holds the row tiles
+// 0 .. min(TI, R * (tj + 1)) - 1 with R = BN / kGramBM, and starts at offset R * tj * (tj + 1) / 2.
+struct GramTiling {
+    int BN;            // columns of an output tile: 128 or 256
+    int R;             // BN / kGramBM
+    int TI, TJ;        // row tiles, column tiles per sample
+    int tiles_per_b;   // visited tiles per sample
+    int n_pad;         // padded token count of one partial-sum slot
+    __host__ __device__ int slots() const { return TJ + TI; }   // rho partial slots per sample: TJ row-side + TI column-side
+};
+
+inline GramTiling make_gram_tiling(int n, int BN) {
+    GramTiling t;
+    t.BN = BN;
+    t.R = BN / kGramBM;
+    t.TI = (n + kGramBM - 1) / kGramBM;
+    t.TJ = (n + BN - 1) / BN;
+    const int last = t.R * t.TJ < t.TI ? t.R * t.TJ : t.TI;
+    t.tiles_per_b = t.TJ > 0 ? t.R * (t.TJ - 1) * t.TJ / 2 + last : 0;
+    t.n_pad = t.TI * kGramBM;
+    return t;
+}
+
+// Tile width the sweeps use for a problem: wide tiles halve the operand traffic per flop, narrow tiles fill
+// the SMs when the problem is small.
+int gram_pick_bn(int B, int n);
+
+struct GramArgs {
+    int B, n, D;
+    int row0, row_end;          // GRAM_SIM: rows [row0, row_end) are produced
+    int metric;                 // 0 cosine, 1 euclid
+    float c2;                   // -(log2 e) / d_c^2
+    float tau2;                 // tau^2; < 0: no spatial test
+    const float* w;             // [B, n] factor multiplying the Gram value (cosine 1/|f|, euclid 1)
+    const float* a;             // [B, n] additive term (cosine 1, euclid |f|^2):  d^2 = a_i + a_j - 2 g w_i w_j
+    const float* rho;           // [B, n]                          (GRAM_DELTA)
+    const float* pos;           // [B, n, 2] or nullptr            (GRAM_DELTA)
+    float* part;                // [B, slots, n_pad] rho partials  (GRAM_RHO)
+    unsigned long long* best;   // [B, n] packed (d2 bits << 32 | index), ~0 = none   (GRAM_DELTA)
+    float* sim_out;             // [B, row_end - row0, n]          (GRAM_SIM)
+    int* status;                // device status word
+};
+
+// Enqueues one sweep.  `tiling` must come from make_gram_tiling(n, gram_pick_bn(B, n)) for the symmetric modes.
+int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream,
+                      bool pdl);
+
+}  // namespace vitcop
