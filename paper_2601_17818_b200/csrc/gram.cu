@@ -8,13 +8,14 @@
 //
 // Symmetry: d_ij = d_ji, so the two sweeps visit only tiles that hold a pair i < j.  Such a pair serves its
 // row token i (a per-thread accumulation along the row) and its column token j (a reduction over the 128
-// rows of the tile, done with a shuffle butterfly inside each warp and a fixed-order combination of the
-// four warps that share a column range).
+// rows of the tile: inside each warp a shuffle butterfly for the sums of Eq. 2 and one redux.sync per column for
+// the minima of Eq. 3, then a fixed-order combination of the four warps that share a column range).
 //
 // One persistent CTA per SM, warp-specialised:
 //   warp 0      TMA producer: feature tiles [128 x 64] and [BN x 64] (128-byte swizzle) into a ring of stages
 //   warp 1      one thread issues tcgen05.mma (M = 128, N = BN, K = 16) into one of two TMEM accumulators
-//   warps 2-9   epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 (its rows) and one half of the columns
+//   warps 2..   epilogue (8 warps for the density sweep, 16 for the delta sweep): warp w reads TMEM lanes
+//               32 * (w % 4) .. + 31 (its rows) and one slice of the columns
 // Every wait is bounded; on expiry the CTA raises an abort flag, all roles leave, TMEM is released and
 // VITCOP_ERR_TIMEOUT is written to the status word.
 #include <cuda.h>
@@ -27,9 +28,10 @@ namespace {
 constexpr int BM = kGramBM;
 constexpr int BK = 64;             // k-block: 64 bf16 = 128 bytes = one 128B-swizzle row
 constexpr int UMMA_K = 16;
-constexpr int kEpiWarps = 8;
-constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kGemmThreads = 64 + kEpiThreads;
+// Column slices an output tile is cut into for the epilogue; every slice is served by four warps (one per
+// TMEM lane quarter).  The delta sweep's epilogue is the heavier one and gets twice the warps.
+__host__ __device__ constexpr int epi_slices(int mode) { return mode == GRAM_DELTA ? 4 : 2; }
+__host__ __device__ constexpr int gemm_threads(int mode) { return 64 + epi_slices(mode) * 128; }
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s give up and leave
 constexpr unsigned long long kDrainLimitNs = 20000000ull;    // bounded waits for this CTA's own copies / MMAs after giving up
 
@@ -132,17 +134,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
     for (int u = 0; u < 32; ++u) v[u] = __uint_as_float(r[u]);
 }
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+template <int THREADS>
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 // Barrier over the epilogue threads that also ORs a predicate: every thread gets the same answer.
+template <int THREADS>
 __device__ __forceinline__ bool epi_bar_or(bool pred) {
     uint32_t out;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, 256, p;\n\t"
+        "bar.red.or.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(out)
-        : "r"((uint32_t)pred)
+        : "r"((uint32_t)pred), "n"(THREADS)
         : "memory");
     return out != 0;
 }
@@ -227,8 +231,9 @@ struct GemmSmem {
     static constexpr int kBBytes = BN * BK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kTileBytes = kStages * kStageBytes;
-    // per column of the tile: w, a, rho, x, y; reduction scratch: 4 x value, 4 x index; per row: value, index
-    static constexpr int kEpiBytes = (5 + 4 + 4) * BN * 4 + 2 * BM * 4;
+    // per column of the tile: w, a, rho, x, y; column reduction scratch: 4 x value, 4 x index;
+    // row reduction scratch: 3 x value, 3 x index
+    static constexpr int kEpiBytes = (5 + 4 + 4) * BN * 4 + (3 + 3) * BM * 4;
     static constexpr int kBarBytes = 256;
     static constexpr int kTotal = 1024 /*alignment slack*/ + kTileBytes + kEpiBytes + kBarBytes;
 };
@@ -239,11 +244,13 @@ constexpr float kInf = __builtin_huge_valf();
 // the kernel
 // ------------------------------------------------------------------------------------------------
 template <int BN, int MODE, int METRIC, bool SPATIAL>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(gemm_threads(MODE), 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const KernelArgs k) {
     using S = GemmSmem<BN>;
     constexpr bool SYM = MODE != GRAM_SIM;
+    constexpr int NS = epi_slices(MODE);
+    constexpr int kEpiThreads = NS * 128;
     const GramArgs& g = k.g;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -256,8 +263,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     float* coly = colx + BN;
     float* colred = coly + BN;                                     // [4][BN]
     int* colidx = reinterpret_cast<int*>(colred + 4 * BN);         // [4][BN]
-    float* rowred = reinterpret_cast<float*>(colidx + 4 * BN);     // [BM]
-    int* rowidx = reinterpret_cast<int*>(rowred + BM);             // [BM]
+    float* rowred = reinterpret_cast<float*>(colidx + 4 * BN);     // [3][BM]
+    int* rowidx = reinterpret_cast<int*>(rowred + 3 * BM);         // [3][BM]
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
     // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], drain
     const uint32_t bar_full = smem_u32(bars);
@@ -278,7 +285,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
-            mbar_init(bar_tempty + 8 * a, kEpiThreads);
+            mbar_init(bar_tempty + 8 * a, kEpiThreads);   // every epilogue thread arrives once per tile
         }
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
@@ -364,12 +371,13 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..9)
-        const int e = threadIdx.x - 64;                    // 0..255
+        // ------------------------------------------------------------------ epilogue (warps 2 ..)
+        const int e = threadIdx.x - 64;                    // 0 .. kEpiThreads - 1
         const int quarter = warp & 3;                      // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;                  // which half of the tile's columns this warp handles
+        const int slice = (warp - 2) >> 2;                 // which slice of the tile's columns this warp handles
         const int rl = quarter * 32 + lane;                // tile-local row == TMEM lane
-        constexpr int kChunks = BN / 64;                   // 32-column chunks per warp
+        constexpr int kSliceCols = BN / NS;
+        constexpr int kChunks = kSliceCols / 32;           // 32-column chunks per warp
         const int rows_out = g.row_end - g.row0;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
@@ -385,16 +393,16 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const size_t bo = (size_t)b * g.n;
 
             // ---- per-column and per-row constants
-            if (e < BN) {
-                const int j = J0 + e;
+            for (int ce = e; ce < BN; ce += kEpiThreads) {
+                const int j = J0 + ce;
                 const bool cv = j < g.n;
-                colw[e] = cv ? g.w[bo + j] : 0.f;
-                if (METRIC == 1) cola[e] = cv ? g.a[bo + j] : 0.f;
+                colw[ce] = cv ? g.w[bo + j] : 0.f;
+                if (METRIC == 1) cola[ce] = cv ? g.a[bo + j] : 0.f;
                 if (MODE == GRAM_DELTA) {
-                    colrho[e] = cv ? g.rho[bo + j] : 0.f;
+                    colrho[ce] = cv ? g.rho[bo + j] : 0.f;
                     if (SPATIAL) {
-                        colx[e] = cv ? g.pos[2 * (bo + j)] : 0.f;
-                        coly[e] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
+                        colx[ce] = cv ? g.pos[2 * (bo + j)] : 0.f;
+                        coly[ce] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
                     }
                 }
             }
@@ -409,7 +417,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // every pair of the tile has i < j < n: no masking needed
             const bool full = SYM && (J0 >= I0 + BM) && (J0 + BN <= g.n);
 
-            epi_bar_sync();
+            epi_bar_sync<kEpiThreads>();
             if (ok) ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
 
@@ -418,7 +426,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int rbest_c = -1;
             if (ok) {
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + half * (BN / 2);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + slice * kSliceCols;
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     float v[32];
@@ -428,7 +436,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         tc_fence_before();
                         mbar_arrive(bar_tempty + 8 * acc);
                     }
-                    const int cl0 = half * (BN / 2) + c * 32;          // tile-local first column of the chunk
+                    const int cl0 = slice * kSliceCols + c * 32;       // tile-local first column of the chunk
+                    const float4* cw4 = reinterpret_cast<const float4*>(colw + cl0);
+                    const float4* ca4 = reinterpret_cast<const float4*>(cola + cl0);
                     if (MODE == GRAM_SIM) {
                         if (row_valid) {
                             float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
@@ -441,11 +451,20 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else if (MODE == GRAM_RHO) {
                         // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
 #pragma unroll
-                        for (int u = 0; u < 32; ++u) {
-                            const float x = v[u] * colw[cl0 + u];
-                            const float base = METRIC == 0 ? 2.f : a_i + cola[cl0 + u];
-                            const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
-                            v[u] = ex2_approx(d2 * g.c2);
+                        for (int q4 = 0; q4 < 8; ++q4) {
+                            const float4 cw = cw4[q4];
+                            float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (METRIC == 1) ca = ca4[q4];
+                            const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                            const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                const int u = 4 * q4 + r;
+                                const float x = v[u] * cwv[r];
+                                const float base = METRIC == 0 ? 2.f : a_i + cav[r];
+                                const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                                v[u] = ex2_approx(d2 * g.c2);
+                            }
                         }
                         if (!full) {
 #pragma unroll
@@ -459,68 +478,87 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const float cs = warp_transpose_reduce<false>(v, lane);
                         colred[quarter * BN + cl0 + lane] = cs;
                     } else {  // GRAM_DELTA, Eq. 3
-                        float kc[32];
+                        const float4* cr4 = reinterpret_cast<const float4*>(colrho + cl0);
+                        const float4* cx4 = reinterpret_cast<const float4*>(colx + cl0);
+                        const float4* cy4 = reinterpret_cast<const float4*>(coly + cl0);
+                        uint32_t kc[32];                   // column-side keys: d^2 >= 0 orders like its bit pattern
+#pragma unroll
+                        for (int q4 = 0; q4 < 8; ++q4) {
+                            const float4 cw = cw4[q4];
+                            const float4 cr = cr4[q4];
+                            float4 ca = make_float4(0.f, 0.f, 0.f, 0.f), cx = ca, cy = ca;
+                            if (METRIC == 1) ca = ca4[q4];
+                            if (SPATIAL) { cx = cx4[q4]; cy = cy4[q4]; }
+                            const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                            const float crv[4] = {cr.x, cr.y, cr.z, cr.w};
+                            const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+                            const float cxv[4] = {cx.x, cx.y, cx.z, cx.w};
+                            const float cyv[4] = {cy.x, cy.y, cy.z, cy.w};
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                const int u = 4 * q4 + r;
+                                const float x = v[u] * cwv[r];
+                                const float base = METRIC == 0 ? 2.f : a_i + cav[r];
+                                float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                                bool usable = true;        // the pair may serve as (child, parent) at all
+                                if (SPATIAL) {
+                                    const float dx = cxv[r] - x_i, dy = cyv[r] - y_i;
+                                    usable = fmaf(dx, dx, dy * dy) <= g.tau2;
+                                }
+                                if (!full) {
+                                    const int j = J0 + cl0 + u;
+                                    usable = usable && j > i && j < g.n && row_valid;
+                                }
+                                if (SPATIAL || !full) d2 = usable ? d2 : kInf;
+                                // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
+                                const bool jd = crv[r] > rho_i;
+                                const float kr = jd ? d2 : kInf;       // j as parent candidate of i (row side)
+                                kc[u] = __float_as_uint(jd ? kInf : d2);   // i as parent candidate of j (column side)
+                                if (kr < rbest) { rbest = kr; rbest_c = cl0 + u; }
+                            }
+                        }
+                        // column side: minimum over this warp's 32 rows and the lowest row that attains it
+                        uint32_t my_min = 0x7f800000u, my_rows = 0;
 #pragma unroll
                         for (int u = 0; u < 32; ++u) {
-                            const float x = v[u] * colw[cl0 + u];
-                            const float base = METRIC == 0 ? 2.f : a_i + cola[cl0 + u];
-                            const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
-                            // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
-                            bool jd = colrho[cl0 + u] > rho_i;
-                            bool id = !jd;
-                            if (SPATIAL) {
-                                const float dx = colx[cl0 + u] - x_i, dy = coly[cl0 + u] - y_i;
-                                const bool near = fmaf(dx, dx, dy * dy) <= g.tau2;
-                                jd = jd && near;
-                                id = id && near;
-                            }
-                            if (!full) {
-                                const int j = J0 + cl0 + u;
-                                const bool pv = j > i && j < g.n && row_valid;
-                                jd = jd && pv;
-                                id = id && pv;
-                            }
-                            const float kr = jd ? d2 : kInf;
-                            kc[u] = id ? d2 : kInf;
-                            if (kr < rbest) { rbest = kr; rbest_c = cl0 + u; }
+                            const uint32_t m = __reduce_min_sync(0xffffffffu, kc[u]);
+                            const uint32_t rows = __ballot_sync(0xffffffffu, kc[u] == m);
+                            if (lane == u) { my_min = m; my_rows = rows; }
                         }
-                        // column side: minimum over this warp's 32 rows, then the lowest row that attains it
-#pragma unroll
-                        for (int u = 0; u < 32; ++u) v[u] = kc[u];
-                        const float cm = warp_transpose_reduce<true>(v, lane);
-                        uint32_t mine = 0;
-#pragma unroll
-                        for (int u = 0; u < 32; ++u) {
-                            const float m = __shfl_sync(0xffffffffu, cm, u);
-                            const uint32_t bal = __ballot_sync(0xffffffffu, kc[u] == m && m < kInf);
-                            if (lane == u) mine = bal;
-                        }
-                        colred[quarter * BN + cl0 + lane] = cm;
-                        colidx[quarter * BN + cl0 + lane] = mine ? I0 + quarter * 32 + (__ffs(mine) - 1) : -1;
+                        colred[quarter * BN + cl0 + lane] = __uint_as_float(my_min);
+                        colidx[quarter * BN + cl0 + lane] =
+                            my_min < 0x7f800000u ? I0 + quarter * 32 + (__ffs(my_rows) - 1) : -1;
                     }
                 }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
 
             if (SYM) {
-                // ---- combine the two column halves of every row and the four row quarters of every column
-                if (half == 1) {
-                    rowred[rl] = MODE == GRAM_RHO ? racc : rbest;
-                    if (MODE == GRAM_DELTA) rowidx[rl] = rbest_c;
+                // ---- combine the four column slices of every row and the four row quarters of every column
+                if (slice > 0) {
+                    rowred[(slice - 1) * BM + rl] = MODE == GRAM_RHO ? racc : rbest;
+                    if (MODE == GRAM_DELTA) rowidx[(slice - 1) * BM + rl] = rbest_c;
                 }
-                epi_bar_sync();
+                epi_bar_sync<kEpiThreads>();
                 if (ok) {
                     const int slot_base = b * k.t.slots();
                     if (MODE == GRAM_RHO) {
-                        if (half == 0 && row_valid)
-                            g.part[((size_t)(slot_base + tj)) * k.t.n_pad + i] = racc + rowred[rl];
-                        if (e < BN && J0 + e < g.n)
-                            g.part[((size_t)(slot_base + k.t.TJ + ti)) * k.t.n_pad + J0 + e] =
-                                ((colred[e] + colred[BN + e]) + colred[2 * BN + e]) + colred[3 * BN + e];
+                        if (slice == 0 && row_valid) {
+#pragma unroll
+                            for (int q = 0; q < NS - 1; ++q) racc += rowred[q * BM + rl];       // fixed order
+                            g.part[((size_t)(slot_base + tj)) * k.t.n_pad + i] = racc;
+                        }
+                        for (int ce = e; ce < BN; ce += kEpiThreads)
+                            if (J0 + ce < g.n)
+                                g.part[((size_t)(slot_base + k.t.TJ + ti)) * k.t.n_pad + J0 + ce] =
+                                    ((colred[ce] + colred[BN + ce]) + colred[2 * BN + ce]) + colred[3 * BN + ce];
                     } else {
-                        if (half == 0 && row_valid) {
-                            const float other = rowred[rl];
-                            if (other < rbest) { rbest = other; rbest_c = rowidx[rl]; }   // tie: the lower column wins
+                        if (slice == 0 && row_valid) {
+#pragma unroll
+                            for (int q = 0; q < NS - 1; ++q) {                             // ascending columns: ties keep the lower one
+                                const float other = rowred[q * BM + rl];
+                                if (other < rbest) { rbest = other; rbest_c = rowidx[q * BM + rl]; }
+                            }
                             if (rbest_c >= 0) {
                                 const unsigned long long packed =
                                     ((unsigned long long)__float_as_uint(rbest) << 32) |
@@ -528,25 +566,26 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 atomicMin(g.best + bo + i, packed);
                             }
                         }
-                        if (e < BN && J0 + e < g.n) {
+                        for (int ce = e; ce < BN; ce += kEpiThreads) {
+                            if (J0 + ce >= g.n) continue;
                             float bk = kInf;
                             int bi = -1;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {                                  // ascending rows: ties keep the lower row
-                                const float kk = colred[q * BN + e];
-                                if (kk < bk) { bk = kk; bi = colidx[q * BN + e]; }
+                                const float kk = colred[q * BN + ce];
+                                if (kk < bk) { bk = kk; bi = colidx[q * BN + ce]; }
                             }
                             if (bi >= 0) {
                                 const unsigned long long packed =
                                     ((unsigned long long)__float_as_uint(bk) << 32) | (unsigned long long)(uint32_t)bi;
-                                atomicMin(g.best + bo + J0 + e, packed);
+                                atomicMin(g.best + bo + J0 + ce, packed);
                             }
                         }
                     }
                 }
             }
             // shared arrays are rewritten for the next tile; all epilogue warps leave together or not at all
-            if (epi_bar_or(!ok)) break;
+            if (epi_bar_or<kEpiThreads>(!ok)) break;
         }
     }
 
@@ -615,7 +654,7 @@ int launch_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(k.total_tiles < num_sms() ? k.total_tiles : num_sms()));
-    cfg.blockDim = dim3(kGemmThreads);
+    cfg.blockDim = dim3(gemm_threads(MODE));
     cfg.dynamicSmemBytes = S::kTotal;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
