@@ -10,7 +10,6 @@ namespace vitcop {
 namespace {
 
 constexpr int kCompactThreads = 256;
-constexpr int kChunk = 8;   // 16-byte pieces a thread holds in registers at once
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;
@@ -25,30 +24,34 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                  : "memory");
 }
 
-// Piece q of the row: [0, dh8) hidden, then H*d8 pieces of K (head-major), then H*d8 pieces of V.
-struct RowMap {
-    const uint4 *hid, *K, *V;
-    uint4 *hid_o, *K_o, *V_o;
-    int dh8, d8, hd8;              // pieces per hidden row, per head row, per all heads
-    int64_t k_head_in, k_head_out;  // pieces between consecutive heads (N*d8, Ncap*d8)
-    __device__ __forceinline__ void locate(int q, const uint4*& src, uint4*& dst) const {
-        if (q < dh8) {
-            src = hid + q;
-            dst = hid_o + q;
-        } else {
-            q -= dh8;
-            const bool isv = q >= hd8;
-            if (isv) q -= hd8;
-            const int h = q / d8, e = q - h * d8;
-            src = (isv ? V : K) + h * k_head_in + e;
-            dst = (isv ? V_o : K_o) + h * k_head_out + e;
+// Copies `total` 16-byte pieces that sit in segments of `seg_len` pieces each (segment s starts at
+// src + s * src_stride / dst + s * dst_stride): one hidden row is a single segment, the K (or V) rows of one
+// token are H segments of d/8 pieces.  Four loads are issued before the first store.
+__device__ __forceinline__ void copy_segments(const uint4* __restrict__ src, uint4* __restrict__ dst, int seg_len,
+                                              int total, int64_t src_stride, int64_t dst_stride, int shift) {
+    for (int q0 = threadIdx.x; q0 < total; q0 += 4 * kCompactThreads) {
+        uint4 v[4];
+        uint4* d[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = q0 + u * kCompactThreads;
+            d[u] = nullptr;
+            if (q < total) {
+                const int sgm = shift >= 0 ? q >> shift : q / seg_len;
+                const int e = q - sgm * seg_len;
+                v[u] = ld_stream(src + sgm * src_stride + e);
+                d[u] = dst + sgm * dst_stride + e;
+            }
         }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (d[u]) st_stream(d[u], v[u]);
     }
-};
+}
 
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, const uint4* __restrict__ V, int H, int N,
-               int d8, int dh8, const int32_t* __restrict__ seq_len, int vis_start,
+               int d8, int dh8, int d8_shift, const int32_t* __restrict__ seq_len, int vis_start,
                const int32_t* __restrict__ vis_len, int vis_len_uniform, const int32_t* __restrict__ keep_idx,
                int keep_stride, const int32_t* __restrict__ n_keep, uint4* __restrict__ hidden_out,
                uint4* __restrict__ K_out, uint4* __restrict__ V_out, int Ncap, int32_t* __restrict__ kept_pos,
@@ -76,46 +79,16 @@ compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, co
     } else src_row = r - nk + nv;
     if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = src_row;
 
-    RowMap m;
-    m.dh8 = hidden ? dh8 : 0;
-    m.d8 = d8 > 0 ? d8 : 1;
-    m.hd8 = H * d8;
-    m.k_head_in = (int64_t)N * d8;
-    m.k_head_out = (int64_t)Ncap * d8;
-    m.hid = hidden ? hidden + ((int64_t)b * N + src_row) * dh8 : nullptr;
-    m.hid_o = hidden ? hidden_out + ((int64_t)b * Ncap + r) * dh8 : nullptr;
-    m.K = K ? K + ((int64_t)b * H * N + src_row) * d8 : nullptr;
-    m.K_o = K ? K_out + ((int64_t)b * H * Ncap + r) * d8 : nullptr;
-    m.V = V ? V + ((int64_t)b * H * N + src_row) * d8 : nullptr;
-    m.V_o = V ? V_out + ((int64_t)b * H * Ncap + r) * d8 : nullptr;
-    // K absent but V present: shift V into K's slot range
-    int total = m.dh8;
-    if (K && V) total += 2 * m.hd8;
-    else if (K) total += m.hd8;
-    else if (V) {
-        m.K = m.V;
-        m.K_o = m.V_o;
-        total += m.hd8;
-    }
-
-    for (int q0 = threadIdx.x; q0 < total; q0 += kCompactThreads * kChunk) {
-        uint4 v[kChunk];
-        uint4* dst[kChunk];
-#pragma unroll
-        for (int u = 0; u < kChunk; ++u) {
-            const int q = q0 + u * kCompactThreads;
-            dst[u] = nullptr;
-            if (q < total) {
-                const uint4* src;
-                m.locate(q, src, dst[u]);
-                v[u] = ld_stream(src);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kChunk; ++u)
-            if (dst[u]) st_stream(dst[u], v[u]);
-    }
-    grid_dependency_launch_dependents();
+    if (hidden)
+        copy_segments(hidden + ((int64_t)b * N + src_row) * dh8, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8, dh8, 0,
+                      0, 31);
+    const int64_t head_in = (int64_t)N * d8, head_out = (int64_t)Ncap * d8;
+    if (K)
+        copy_segments(K + ((int64_t)b * H * N + src_row) * d8, K_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
+                      head_in, head_out, d8_shift);
+    if (V)
+        copy_segments(V + ((int64_t)b * H * N + src_row) * d8, V_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
+                      head_in, head_out, d8_shift);
 }
 
 }  // namespace
@@ -125,6 +98,10 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
                    const int32_t* keep_idx, int keep_stride, const int32_t* n_keep, void* hidden_out, void* K_out,
                    void* V_out, int Ncap, int32_t* kept_pos, int32_t* out_len, cudaStream_t stream, bool pdl) {
     if (B <= 0) return VITCOP_OK;
+    const int d8 = d / 8;
+    int d8_shift = -1;                                    // log2(d / 8) when that is a power of two
+    if (d8 > 0 && (d8 & (d8 - 1)) == 0)
+        for (d8_shift = 0; (1 << d8_shift) < d8; ++d8_shift) {}
     cudaLaunchConfig_t cfg = {};
     // rows past min(N, Ncap) cannot exist; one extra CTA row keeps out_len written when Ncap == 0
     const int rows = Ncap > 0 ? Ncap : 1;
@@ -139,7 +116,7 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
     KernelTimeScope timed("compact_kernel", stream);
     return record_cuda(cudaLaunchKernelEx(
         &cfg, compact_kernel, static_cast<const uint4*>(hidden), static_cast<const uint4*>(K),
-        static_cast<const uint4*>(V), H, N, d / 8, Dh / 8, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
+        static_cast<const uint4*>(V), H, N, d / 8, Dh / 8, d8_shift, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
         keep_stride, n_keep, static_cast<uint4*>(hidden_out), static_cast<uint4*>(K_out), static_cast<uint4*>(V_out),
         Ncap, kept_pos, out_len));
 }

@@ -108,7 +108,7 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
     int32_t* centres = reinterpret_cast<int32_t*>(fin_smem + (size_t)n * 8 + (((size_t)n + 15) & ~(size_t)15));
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t s_digit, s_krem;
+    __shared__ uint32_t s_digit, s_krem, s_whole;
 
     grid_dependency_launch_dependents();
     grid_dependency_wait();
@@ -176,12 +176,20 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
                 if (excl < krem && krem <= incl) {
                     s_digit = (uint32_t)tid;
                     s_krem = krem - excl;
+                    s_whole = (c == krem - excl) ? 1u : 0u;         // the whole bin is wanted
                 }
             }
             __syncthreads();
             prefix |= (unsigned long long)s_digit << shift;
             krem = s_krem;
+            const bool whole = s_whole != 0;
             __syncthreads();
+            if (whole) {
+                // every key that shares the prefix found so far is selected: no need to resolve lower digits
+                prefix |= (1ull << shift) - 1ull;
+                krem = 0xFFFFFFFFu;
+                break;
+            }
         }
         T = prefix;
     }

@@ -33,6 +33,8 @@ __device__ __forceinline__ void sq_acc(const uint4& v, float& a0, float& a1) {
 }
 
 // Strides are in units of 16 bytes (8 elements).
+// The loads of head batch k + 1 are issued before the squares of batch k are accumulated, so that every
+// thread always has UNROLL 16-byte requests in flight and the batches do not run in lock step.
 template <int LPR, int UNROLL>
 __global__ void __launch_bounds__(kKnormThreads)
 knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh, int64_t sn, int vis_start,
@@ -48,15 +50,23 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
         const uint4* base = K + b * sb + (int64_t)(vis_start + i) * sn;
         for (int c = sub; c < d8; c += LPR) {
             const uint4* p = base + c;
-            int h = 0;
-            for (; h + UNROLL <= H; h += UNROLL) {
-                uint4 v[UNROLL];
+            const int full = H / UNROLL * UNROLL;
+            if (full > 0) {
+                uint4 cur[UNROLL], nxt[UNROLL];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(p + (int64_t)(h + u) * sh);
+                for (int u = 0; u < UNROLL; ++u) cur[u] = ld_stream(p + (int64_t)u * sh);
+                for (int h = UNROLL; h < full; h += UNROLL) {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) sq_acc(v[u], a0, a1);
+                    for (int u = 0; u < UNROLL; ++u) nxt[u] = ld_stream(p + (int64_t)(h + u) * sh);
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) sq_acc(cur[u], a0, a1);
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) cur[u] = nxt[u];
+                }
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) sq_acc(cur[u], a0, a1);
             }
-            for (; h < H; ++h) {
+            for (int h = full; h < H; ++h) {
                 const uint4 v = ld_stream(p + (int64_t)h * sh);
                 sq_acc(v, a0, a1);
             }
@@ -66,6 +76,8 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
 #pragma unroll
     for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (i < nv && sub == 0) score[(int64_t)b * Nv_cap + i] = sqrtf(acc);
+    // Only now may the next kernel's CTAs be scheduled: released earlier they would sit on the SMs waiting for
+    // this grid while its own remaining CTAs queue behind them.
     grid_dependency_launch_dependents();
 }
 
@@ -80,18 +92,27 @@ int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t s
     if (span <= 0) return VITCOP_OK;
     const uint4* Kp = static_cast<const uint4*>(K);
     const int64_t sb = stride_b / 8, sh = stride_h / 8, sn = stride_n / 8;
+    int rc = VITCOP_OK;
     auto go = [&](auto kern, int lpr) {
         const int tok = kKnormThreads / lpr;
-        dim3 grid((span + tok - 1) / tok, B);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((span + tok - 1) / tok, B);
+        cfg.blockDim = dim3(kKnormThreads);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl_allowed(true) ? 1 : 0;
         KernelTimeScope timed("knorm_kernel", stream);
-        kern<<<grid, kKnormThreads, 0, stream>>>(Kp, H, d8, sb, sh, sn, vis_start, vis_len, vis_len_uniform, score,
-                                                  Nv_cap);
+        rc = record_cuda(cudaLaunchKernelEx(&cfg, kern, Kp, H, d8, sb, sh, sn, vis_start, vis_len, vis_len_uniform,
+                                            score, Nv_cap));
     };
     if (d8 >= 16) go(knorm_kernel<16, 8>, 16);
     else if (d8 >= 8) go(knorm_kernel<8, 8>, 8);
     else if (d8 >= 4) go(knorm_kernel<4, 8>, 4);
     else go(knorm_kernel<1, 8>, 1);
-    return record_cuda(cudaGetLastError());
+    return rc;
 }
 
 }  // namespace vitcop

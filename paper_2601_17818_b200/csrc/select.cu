@@ -72,7 +72,7 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     uint32_t* keys = smem_u32;
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_sums[kSelWarps];
-    __shared__ uint32_t s_digit, s_krem;
+    __shared__ uint32_t s_digit, s_krem, s_whole;
 
     grid_dependency_wait();
     const int b = blockIdx.x;
@@ -125,12 +125,20 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
                 if (excl < krem && krem <= incl) {
                     s_digit = (uint32_t)tid;
                     s_krem = krem - excl;
+                    s_whole = (c == krem - excl) ? 1u : 0u;         // the whole bin is wanted
                 }
             }
             __syncthreads();
             prefix |= s_digit << shift;
             krem = s_krem;
+            const bool whole = s_whole != 0;
             __syncthreads();
+            if (whole) {
+                // every key that shares the prefix found so far is kept: no need to resolve lower digits
+                prefix |= (1u << shift) - 1u;
+                krem = 0xFFFFFFFFu;
+                break;
+            }
         }
         T = prefix;
     }
@@ -162,6 +170,94 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     grid_dependency_launch_dependents();
 }
 
+// ------------------------------------------------------------------------------------------ block sort
+// Bitonic sort of P = E * T 64-bit keys held E per thread by the first T threads of the CTA (T a multiple of
+// 32, P a power of two), blocked: key p = t * E + e sits in slot e of thread t.  Compare-exchange partners at
+// distance j < E are two slots of one thread; at distance j = m * E they are the same slot of threads t and
+// t ^ m -- two lanes of a warp for m < 32 (shuffles), two warps otherwise (exchanged through `sm`, P keys).
+// All threads of the CTA must call; on return sm[p] holds the ascending order.
+template <int E, int J>
+__device__ __forceinline__ void bitonic_local(unsigned long long (&r)[E], int base, int k) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        if ((e & J) == 0 && (e | J) < E) {
+            const bool up = ((base + e) & k) == 0;
+            const unsigned long long a = r[e], c = r[e | J];
+            if ((a > c) == up) { r[e] = c; r[e | J] = a; }
+        }
+    }
+}
+
+// Barrier over the first `count` threads of the CTA (a multiple of 32), leaving the other warps out.
+__device__ __forceinline__ void active_bar_sync(int count) { asm volatile("bar.sync 1, %0;" ::"r"(count) : "memory"); }
+
+template <int E>
+__device__ void block_bitonic_sort(unsigned long long (&r)[E], unsigned long long* sm, int T) {
+    const int t = threadIdx.x;
+    const int P = E * T;
+    const int base = t * E;
+    // Warps that hold no keys skip the network altogether: spinning through its empty iterations would take
+    // issue slots away from the few warps that do the work when P is small.
+    if (t < T) {
+        for (int k = 2; k <= P; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                if (j < E) {
+                    if (j == 1) bitonic_local<E, 1>(r, base, k);
+                    else if (j == 2) bitonic_local<E, 2>(r, base, k);
+                    else if (j == 4) bitonic_local<E, 4>(r, base, k);
+                    else bitonic_local<E, 8>(r, base, k);
+                    continue;
+                }
+                const int m = j / E;                       // partner thread is t ^ m
+                const bool lower = (t & m) == 0;
+                const bool up = (base & k) == 0;           // k > j >= E: the same for all slots of a thread
+                const bool want_min = lower == up;
+                if (m < 32) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const unsigned long long o = __shfl_xor_sync(0xffffffffu, r[e], m);
+                        r[e] = (want_min == (o < r[e])) ? o : r[e];
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) sm[e * T + t] = r[e];
+                    active_bar_sync(T);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const unsigned long long o = sm[e * T + (t ^ m)];
+                        r[e] = (want_min == (o < r[e])) ? o : r[e];
+                    }
+                    active_bar_sync(T);
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) sm[base + e] = r[e];
+    }
+    __syncthreads();
+}
+
+// Loads the composite keys (label, score key, index) of one sequence, padded with ~0 up to P, and sorts them.
+template <int E>
+__device__ void sort_composites(const float* __restrict__ score, const int32_t* __restrict__ label, int n, int T,
+                                unsigned long long* comp) {
+    unsigned long long r[E];
+    const int t = threadIdx.x;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int i = t * E + e;
+        unsigned long long c = ~0ull;
+        if (t < T && i < n) {
+            uint32_t lab = (uint32_t)label[i];
+            if (lab >= (uint32_t)n) lab = (uint32_t)n - 1;          // out-of-range labels are clamped, never indexed
+            c = ((unsigned long long)lab << 48) | ((unsigned long long)order_key(score[i], 0) << 16) |
+                (unsigned long long)i;
+        }
+        r[e] = c;
+    }
+    block_bitonic_sort<E>(r, comp, T);
+}
+
 // ------------------------------------------------------------------------------------------ quota
 // Shared memory: comp[P] (uint64), cstart[n] and csize[n] (uint16, indexed by label value), keep[n] (uint8).
 __global__ void __launch_bounds__(kSelThreads)
@@ -186,36 +282,11 @@ select_quota_kernel(const float* __restrict__ score, const int32_t* __restrict__
     keep_idx += (int64_t)b * keep_stride;
     if (keep_mask) keep_mask += (int64_t)b * Nv_cap;
 
-    int P = 1;
+    int P = 256;                                          // at least one warp of 8 keys per thread
     while (P < n) P <<= 1;
-    for (int i = tid; i < P; i += kSelThreads) {
-        unsigned long long c = ~0ull;
-        if (i < n) {
-            uint32_t lab = (uint32_t)label[i];
-            if (lab >= (uint32_t)n) lab = (uint32_t)n - 1;          // out-of-range labels are clamped, never indexed
-            c = ((unsigned long long)lab << 48) | ((unsigned long long)order_key(score[i], 0) << 16) |
-                (unsigned long long)i;
-        }
-        comp[i] = c;
-    }
     for (int i = tid; i < n; i += kSelThreads) keepf[i] = 0;
-    __syncthreads();
-
-    for (int kk = 2; kk <= P; kk <<= 1) {
-        for (int j = kk >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (P >> 1); t += kSelThreads) {
-                const int i = 2 * t - (t & (j - 1));
-                const int p = i + j;
-                const unsigned long long a = comp[i], c = comp[p];
-                const bool up = (i & kk) == 0;
-                if ((a > c) == up) {
-                    comp[i] = c;
-                    comp[p] = a;
-                }
-            }
-            __syncthreads();
-        }
-    }
+    if (P <= 8 * kSelThreads) sort_composites<8>(score, label, n, P / 8, comp);
+    else sort_composites<16>(score, label, n, P / 16, comp);
 
     // cluster heads / tails in the sorted order
     uint32_t heads_here = 0;
@@ -288,7 +359,7 @@ int launch_select(const float* score, const int32_t* label, int B, const int32_t
         return record_cuda(cudaLaunchKernelEx(&cfg, select_plain_kernel, score, vis_len, vis_len_uniform, Nv_cap,
                                               largest, budget, keep_idx, keep_stride, n_keep, keep_mask));
     }
-    int P = 1;
+    int P = 256;
     while (P < cap) P <<= 1;
     const size_t smem = (size_t)P * 8 + (size_t)cap * (2 + 2 + 1) + 16;
     if (smem > 48 * 1024) {
