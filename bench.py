@@ -260,6 +260,29 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
     return out
 
 
+def host_inputs(w, torch):
+    """Seeded inputs of one workload as pinned host tensors."""
+    feat_b, pos = W.make_features(w), W.make_positions(w)
+    K_b, V_b = W.make_kv(w, 0, w.Nv)
+    hid_b = W.make_hidden(w)
+    bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+    return {"feat": bf(feat_b), "pos": torch.from_numpy(pos.copy()).pin_memory(), "K": bf(K_b), "V": bf(V_b),
+            "hidden": bf(hid_b)}
+
+
+def kernel_times(vb, torch, st, flush, reps):
+    """Per-kernel (launches, total ms) of `reps` steps, from the library's own CUDA-event brackets."""
+    for _ in range(3):
+        flush.zero_()
+        st.run()
+    torch.cuda.synchronize()
+    vb.vitcop_kernel_timing_begin()
+    for _ in range(reps):
+        flush.zero_()
+        st.run()
+    return vb.vitcop_kernel_timing_end()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -279,14 +302,7 @@ def run_ours(args):
     peaks = measured_peaks()
 
     # host inputs (pinned) ---------------------------------------------------------------------------
-    feat_b, pos = W.make_features(w), W.make_positions(w)
-    K_b, V_b = W.make_kv(w, 0, w.Nv)
-    hid_b = W.make_hidden(w)
-    host = {"feat": torch.from_numpy(feat_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
-            "pos": torch.from_numpy(pos).pin_memory(),
-            "K": torch.from_numpy(K_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
-            "V": torch.from_numpy(V_b.view(np.int16)).view(torch.bfloat16).pin_memory(),
-            "hidden": torch.from_numpy(hid_b.view(np.int16)).view(torch.bfloat16).pin_memory()}
+    host = host_inputs(w, torch)
     st = Step(w, torch, vb, dev)
     st.upload(host, non_blocking=False)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)     # > 4x the 126 MB L2
@@ -332,16 +348,13 @@ def run_ours(args):
 
     # per-kernel device times: the library brackets each of its kernels with CUDA events on the stream ----
     n_kt = max(10, min(args.steps, 50))
-    for _ in range(3):
-        flush.zero_()
-        st.run()
-    torch.cuda.synchronize()
-    vb.vitcop_kernel_timing_begin()
-    for _ in range(n_kt):
-        flush.zero_()
-        st.run()
-    per_kernel = vb.vitcop_kernel_timing_end()
+    per_kernel = kernel_times(vb, torch, st, flush, n_kt)
     kernels = kernel_rooflines(w, nk_total, per_kernel, peaks)
+    # what a pair of event records adds to a kernel it brackets, measured on an empty-ish kernel: the per-kernel
+    # times above (and the roofline fractions computed from them) include it, nothing is subtracted
+    tiny = torch.zeros(32, device=dev)
+    t_br = timed(lambda: tiny.zero_(), 20, 3)
+    bracket_us = float(np.median(t_br) * 1e3)
     launches_per_step = sum(v[0] for v in per_kernel.values()) // n_kt
     dom = max(per_kernel, key=lambda k: per_kernel[k][1])
     roofline = {"kernel": dom}
@@ -349,7 +362,8 @@ def run_ours(args):
     roofline.update(peak_source=peaks["source"] + (" burst" if kernels[dom].get("bound") == "tensor" else " copy"),
                     us_per_launch=kernels[dom]["us_per_launch"],
                     algorithmic_units_per_launch=kernels[dom].get("algorithmic_units_per_launch"),
-                    share_of_step=per_kernel[dom][1] / sum(v[1] for v in per_kernel.values()))
+                    share_of_step=per_kernel[dom][1] / sum(v[1] for v in per_kernel.values()),
+                    event_bracket_overhead_us=bracket_us)
 
     # per-API-call times (same protocol as the step) -----------------------------------------------------------
     score = torch.empty((w.B, w.Nv), dtype=torch.float32, device=dev)
@@ -402,6 +416,26 @@ def run_ours(args):
                "sample": f"the first {sample_B} of {w.B} sequences of workload {w.name}, whole hot path, "
                          f"{passes} passes in {secs:.1f} s"}
 
+    # the larger workloads, same protocol, fewer steps (context for the fractions: c1 is latency-bound) --------
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_workloads:
+        others = {}
+        for name in ("c2", "c3", "c4"):
+            wo = W.workload(name)
+            so = Step(wo, torch, vb, dev)
+            so.upload(host_inputs(wo, torch), non_blocking=False)
+            t = timed(so.run, 20, 3)
+            nko = so.nkeep.cpu().numpy()
+            pk = kernel_times(vb, torch, so, flush, 10)
+            ks = kernel_rooflines(wo, int(nko.sum()), pk, peaks)
+            others[name] = {"us_per_step_median": float(np.median(t) * 1e3),
+                            "value": float((wo.Nv - nko).sum() / (np.median(t) * 1e-3)), "unit": UNIT,
+                            "config": config_of(wo),
+                            "kernels": {k: {a: v[a] for a in ("us_per_launch", "bound", "achieved", "unit", "frac")
+                                            if a in v} for k, v in ks.items()}}
+            del so
+            torch.cuda.empty_cache()
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -412,6 +446,7 @@ def run_ours(args):
                                 l2="flushed (512 MiB memset) before every timed step", sharding="replicas only"),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels, "stages": stage,
+            "other_workloads": others,
             "us_per_step_median": float(np.median(t_step) * 1e3),
         }
         print(json.dumps(line))
@@ -427,6 +462,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the c2-c4 summary (N = 1 only)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="length of the CPU-oracle timing leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
