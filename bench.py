@@ -38,6 +38,10 @@ UNIT = "tokens/s"
 # (bytes per launch on the bench workload, sha1 of the kernel's source file when the counters were taken).
 # A kernel whose source changed since reports traffic null.
 NCU_TRAFFIC = {
+    "gram_tc_kernel<delta>": (19137024, "602bd8329f76"),
+    "gram_tc_kernel<rho>": (18940416, "602bd8329f76"),
+    "knorm_kernel": (75522560 + 1190400, "3e4bfc525f97"),
+    "compact_kernel": (33737728 + 1013760, "619ac324b74f"),
 }
 
 
@@ -239,8 +243,8 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
         "gram_tc_kernel<rho>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
         "gram_tc_kernel<delta>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
     }
-    src = {"knorm_kernel": "knorm.cu", "compact_kernel": "compact.cu", "gram_tc_kernel<rho>": "filter.cu",
-           "gram_tc_kernel<delta>": "filter.cu"}
+    src = {"knorm_kernel": "knorm.cu", "compact_kernel": "compact.cu", "gram_tc_kernel<rho>": "gram.cu",
+           "gram_tc_kernel<delta>": "gram.cu"}
     out = {}
     for name, (launches, ms) in per_kernel.items():
         us = ms * 1e3 / max(launches, 1)
@@ -251,8 +255,8 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
                 ach, peak, unit = units / (us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
             else:
                 ach, peak, unit = units / (us * 1e-6) / 1e12, peaks["bf16_tflops"], "TFLOP/s"
-            traffic = None
-            if name in NCU_TRAFFIC and NCU_TRAFFIC[name][1] == source_sha(src[name]):
+            traffic = None                      # the counters were taken on workload c1 only
+            if w.name == "c1" and name in NCU_TRAFFIC and NCU_TRAFFIC[name][1] == source_sha(src[name]):
                 traffic = NCU_TRAFFIC[name][0]
             e.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=traffic,
                      algorithmic_units_per_launch=units)
