@@ -2,7 +2,8 @@
 //
 // Pipeline (one stream, no host synchronisation; consecutive kernels overlap through programmatic dependent
 // launch, each waiting for its predecessor before it reads what that one wrote):
-//   1. row_stats_kernel       |f_i|^2 in fp32 -> per-token factors (cosine: 1/|f_i|; euclid: |f_i|^2)
+//   1. Gram sweep, GRAM_DIAG  the diagonal tiles only: g_ii -> per-token factors (cosine: 1/sqrt(g_ii);
+//                             euclid: g_ii), from the same tensor-core arithmetic as every g_ij
 //   2. Gram sweep, GRAM_RHO   Gram tiles on the tensor cores (gram.cu); the epilogue turns each tile into
 //                             squared distances, exp(-(d/d_c)^2) and partial sums of Eq. 2 per tile
 //   3. rho_reduce_kernel      fixed-order sum of the partials -> rho (bit-reproducible)
@@ -20,38 +21,6 @@ constexpr int BM = kGramBM;
 // ------------------------------------------------------------------------------------------------
 // small kernels
 // ------------------------------------------------------------------------------------------------
-// One warp per token: |f|^2 in fp32, then the epilogue factors.  Also resets the packed minima.
-__global__ void row_stats_kernel(const uint4* __restrict__ feat, int total_rows, int D8, int metric,
-                                 float* __restrict__ w, float* __restrict__ a, unsigned long long* __restrict__ best) {
-    grid_dependency_launch_dependents();
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= total_rows) return;
-    const uint4* p = feat + (size_t)row * D8;
-    float s0 = 0.f, s1 = 0.f;
-    for (int c = lane; c < D8; c += 32) {
-        const uint4 v = p[c];
-        float x;
-        x = bf16lo(v.x); s0 = fmaf(x, x, s0);  x = bf16hi(v.x); s1 = fmaf(x, x, s1);
-        x = bf16lo(v.y); s0 = fmaf(x, x, s0);  x = bf16hi(v.y); s1 = fmaf(x, x, s1);
-        x = bf16lo(v.z); s0 = fmaf(x, x, s0);  x = bf16hi(v.z); s1 = fmaf(x, x, s1);
-        x = bf16lo(v.w); s0 = fmaf(x, x, s0);  x = bf16hi(v.w); s1 = fmaf(x, x, s1);
-    }
-    float s = s0 + s1;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    if (lane == 0) {
-        if (metric == 0) {
-            w[row] = s > 0.f ? 1.0f / sqrtf(s) : 0.f;
-            a[row] = 1.f;
-        } else {
-            w[row] = 1.f;
-            a[row] = s;
-        }
-        if (best) best[row] = ~0ull;
-    }
-}
-
 // rho[b,i] = sum of the partials of the tiles that hold token i, in a fixed order (reproducible bits):
 // the row-side slots of the column tiles that pair row tile i / 128 with later tokens, then the column-side
 // slots of the row tiles that pair column tile i / BN with earlier tokens.
@@ -312,16 +281,6 @@ void pdl_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 grid, d
     cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
 }
 
-int launch_row_stats(const void* feat, int rows, int D, int metric, float* w, float* a, unsigned long long* best,
-                     cudaStream_t stream) {
-    // first kernel of a call: launched without programmatic overlap, so everything queued before the call
-    // (the producer of the features included) has completed when it starts
-    KernelTimeScope timed("row_stats_kernel", stream);
-    row_stats_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(feat), rows, D / 8, metric, w, a,
-                                                         best);
-    return record_cuda(cudaGetLastError());
-}
-
 }  // namespace
 
 size_t filter_workspace_bytes(int B, int n, int D) {
@@ -344,17 +303,19 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     unsigned long long* best = reinterpret_cast<unsigned long long*>(ws + l.off_best);
     float* part = reinterpret_cast<float*>(ws + l.off_part);
 
-    int rc = launch_row_stats(feat, B * n, D, p.metric, w, a, best, stream);
-    if (rc != VITCOP_OK) return rc;
-
     const GramTiling tiling = make_gram_tiling(n, gram_pick_bn(B, n));
     GramArgs g = {};
     g.B = B; g.n = n; g.D = D; g.row0 = 0; g.row_end = n; g.metric = p.metric;
     g.c2 = -1.4426950408889634f / (p.d_c * p.d_c);
     g.tau2 = (p.tau >= 0.f && pos) ? p.tau * p.tau : -1.f;
     g.w = w; g.a = a; g.rho = rho; g.pos = pos; g.part = part; g.best = best;
+    g.w_out = w; g.a_out = a;
     g.sim_out = nullptr; g.status = reinterpret_cast<int*>(ws);
 
+    // first kernel of the call: launched without programmatic overlap, so everything queued before the call
+    // (the producer of the features included) has completed when it starts
+    int rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
+    if (rc != VITCOP_OK) return rc;
     rc = launch_gram_sweep(GRAM_RHO, feat, g, tiling, stream, true);
     if (rc != VITCOP_OK) return rc;
     {
@@ -388,12 +349,12 @@ int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, in
     char* ws = static_cast<char*>(workspace);
     float* w = reinterpret_cast<float*>(ws + kStatusBytes);
     float* a = reinterpret_cast<float*>(ws + kStatusBytes + align_up((size_t)B * n * 4, 256));
-    int rc = launch_row_stats(feat, B * n, D, metric, w, a, nullptr, stream);
-    if (rc != VITCOP_OK) return rc;
     GramArgs g = {};
     g.B = B; g.n = n; g.D = D; g.row0 = row_begin; g.row_end = row_end; g.metric = metric;
     g.c2 = 0.f; g.tau2 = -1.f;
-    g.w = w; g.a = a; g.sim_out = out; g.status = reinterpret_cast<int*>(ws);
+    g.w = w; g.a = a; g.w_out = w; g.a_out = a; g.sim_out = out; g.status = reinterpret_cast<int*>(ws);
+    int rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
+    if (rc != VITCOP_OK) return rc;
     return launch_gram_sweep(GRAM_SIM, feat, g, make_gram_tiling(n, 128), stream, true);
 }
 

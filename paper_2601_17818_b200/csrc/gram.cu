@@ -181,10 +181,14 @@ struct KernelArgs {
     long long total_tiles;
 };
 
-template <int BN, bool SYM>
+template <int BN, bool SYM, bool DIAG = false>
 __device__ __forceinline__ void decode_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
     b = (int)(t / k.t.tiles_per_b);
     const int r = (int)(t - (long long)b * k.t.tiles_per_b);
+    if (DIAG) {
+        ti = tj = r;
+        return;
+    }
     if (!SYM) {
         ti = r / k.t.TJ;
         tj = r - ti * k.t.TJ;
@@ -248,7 +252,8 @@ __global__ void __launch_bounds__(gemm_threads(MODE), 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const KernelArgs k) {
     using S = GemmSmem<BN>;
-    constexpr bool SYM = MODE != GRAM_SIM;
+    constexpr bool SYM = MODE == GRAM_RHO || MODE == GRAM_DELTA;
+    constexpr bool DIAG = MODE == GRAM_DIAG;            // BN == BM: a diagonal tile multiplies the row block by itself
     constexpr int NS = epi_slices(MODE);
     constexpr int kEpiThreads = NS * 128;
     const GramArgs& g = k.g;
@@ -316,14 +321,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
                 int b, ti, tj;
-                decode_tile<BN, SYM>(k, t, b, ti, tj);
+                decode_tile<BN, SYM, DIAG>(k, t, b, ti, tj);
                 const int I0 = g.row0 + ti * BM, J0 = tj * BN;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = tiles + stage * S::kStageBytes;
-                    mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
+                    mbar_expect_tx(bar_full + 8 * stage, DIAG ? S::kABytes : S::kStageBytes);
                     tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
-                    tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
+                    if (!DIAG) tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
                     issued |= 1u << stage;
                     issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
@@ -350,7 +355,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles + stage * S::kStageBytes;
-                    const uint64_t da = umma_desc_k128(sa), db = umma_desc_k128(sa + S::kABytes);
+                    const uint64_t da = umma_desc_k128(sa), db = DIAG ? da : umma_desc_k128(sa + S::kABytes);
 #pragma unroll
                     for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                         // advancing 16 elements (32 bytes) along K inside the swizzle row: +2 in address units
@@ -386,14 +391,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             int b, ti, tj;
-            decode_tile<BN, SYM>(k, t, b, ti, tj);
+            decode_tile<BN, SYM, DIAG>(k, t, b, ti, tj);
             const int I0 = g.row0 + ti * BM, J0 = tj * BN;
             const int i = I0 + rl;
             const bool row_valid = SYM ? (i < g.n) : (i < g.row_end);
             const size_t bo = (size_t)b * g.n;
 
             // ---- per-column and per-row constants
-            for (int ce = e; ce < BN; ce += kEpiThreads) {
+            for (int ce = e; ce < BN && !DIAG; ce += kEpiThreads) {
                 const int j = J0 + ce;
                 const bool cv = j < g.n;
                 colw[ce] = cv ? g.w[bo + j] : 0.f;
@@ -406,7 +411,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
             }
-            const float w_i = row_valid ? g.w[bo + i] : 0.f;
+            const float w_i = (row_valid && !DIAG) ? g.w[bo + i] : 0.f;
             const float a_i = METRIC == 1 ? (row_valid ? g.a[bo + i] : 0.f) : 1.f;
             const float m2w_i = -2.f * w_i;
             float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
@@ -439,7 +444,20 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int cl0 = slice * kSliceCols + c * 32;       // tile-local first column of the chunk
                     const float4* cw4 = reinterpret_cast<const float4*>(colw + cl0);
                     const float4* ca4 = reinterpret_cast<const float4*>(cola + cl0);
-                    if (MODE == GRAM_SIM) {
+                    if (MODE == GRAM_DIAG) {
+                        // g_ii sits in column rl of row rl: the chunk that starts at this warp's first row
+                        if (cl0 == quarter * 32 && row_valid) {
+                            float gii = 0.f;
+#pragma unroll
+                            for (int u = 0; u < 32; ++u) gii = (u == lane) ? v[u] : gii;
+                            // The squared norm comes from the same tensor-core arithmetic as every g_ij, so the
+                            // rounding of the accumulation cancels in s_ij = g_ij / sqrt(g_ii g_jj) where it
+                            // matters: near-duplicates (s -> 1, d^2 = 2 - 2 s -> 0); exact duplicates give s = 1.
+                            g.w_out[bo + i] = METRIC == 0 ? (gii > 0.f ? 1.0f / sqrtf(gii) : 0.f) : 1.f;
+                            g.a_out[bo + i] = METRIC == 0 ? 1.f : gii;
+                            if (g.best) g.best[bo + i] = ~0ull;
+                        }
+                    } else if (MODE == GRAM_SIM) {
                         if (row_valid) {
                             float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
 #pragma unroll
@@ -663,7 +681,8 @@ int launch_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k
     cfg.attrs = attr;
     cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
     KernelTimeScope timed(MODE == GRAM_RHO ? "gram_tc_kernel<rho>"
-                                           : MODE == GRAM_DELTA ? "gram_tc_kernel<delta>" : "gram_tc_kernel<sim>",
+                          : MODE == GRAM_DELTA ? "gram_tc_kernel<delta>"
+                          : MODE == GRAM_DIAG ? "gram_tc_kernel<diag>" : "gram_tc_kernel<sim>",
                           stream);
     return record_cuda(cudaLaunchKernelEx(&cfg, kern, ma, mb, k));
 }
@@ -683,6 +702,10 @@ int launch_bn(int mode, const CUtensorMap& ma, const CUtensorMap& mb, const Kern
                               : launch_one<BN, GRAM_DELTA, 0, true>(ma, mb, k, stream, pdl);
             return euclid ? launch_one<BN, GRAM_DELTA, 1, false>(ma, mb, k, stream, pdl)
                           : launch_one<BN, GRAM_DELTA, 0, false>(ma, mb, k, stream, pdl);
+        case GRAM_DIAG:
+            if (BN != BM) return VITCOP_ERR_INVALID_ARG;
+            return euclid ? launch_one<BM, GRAM_DIAG, 1, false>(ma, mb, k, stream, pdl)
+                          : launch_one<BM, GRAM_DIAG, 0, false>(ma, mb, k, stream, pdl);
         default:
             return euclid ? launch_one<BN, GRAM_SIM, 1, false>(ma, mb, k, stream, pdl)
                           : launch_one<BN, GRAM_SIM, 0, false>(ma, mb, k, stream, pdl);
@@ -711,6 +734,7 @@ int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const Gr
     } else {
         k.g.row0 = 0;
         k.g.row_end = args.n;
+        if (mode == GRAM_DIAG) k.t.tiles_per_b = k.t.TI;        // one tile per 128-row block (tiling.BN == 128)
     }
     k.total_tiles = (long long)args.B * k.t.tiles_per_b;
     if (k.total_tiles <= 0) return VITCOP_OK;

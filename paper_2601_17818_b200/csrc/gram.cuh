@@ -7,7 +7,8 @@ namespace vitcop {
 
 constexpr int kGramBM = 128;   // rows of an output tile (UMMA M)
 
-enum GramMode { GRAM_RHO = 0, GRAM_DELTA = 1, GRAM_SIM = 2 };
+// GRAM_DIAG visits only the diagonal tiles and turns g_ii into the per-token factors w and a.
+enum GramMode { GRAM_RHO = 0, GRAM_DELTA = 1, GRAM_SIM = 2, GRAM_DIAG = 3 };
 
 // Tiling of the symmetric sweeps (GRAM_RHO, GRAM_DELTA).  Only tiles that hold a pair (i, j) with i < j are
 // visited; a pair contributes to its row token i ("row side") and to its column token j ("column side").
@@ -51,6 +52,8 @@ struct GramArgs {
     float* part;                // [B, slots, n_pad] rho partials  (GRAM_RHO)
     unsigned long long* best;   // [B, n] packed (d2 bits << 32 | index), ~0 = none   (GRAM_DELTA)
     float* sim_out;             // [B, row_end - row0, n]          (GRAM_SIM)
+    float* w_out;               // [B, n] factors written by GRAM_DIAG (best, if given, is reset to ~0 as well)
+    float* a_out;               // [B, n]
     int* status;                // device status word
 };
 
