@@ -48,6 +48,9 @@ def lib() -> C.CDLL:
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.oracle_cr_int.restype = C.c_double
+        _lib.oracle_flops_layer.restype = C.c_double
+        _lib.oracle_visual_tokens_at_layer.restype = C.c_double
+        _lib.oracle_flops_vitcop.restype = C.c_double
     return _lib
 
 
@@ -222,6 +225,50 @@ def stage_count(m: int, pi: float) -> int:
 
 def cr_int(pi1: float, pi2: float, pi3: float, l_s: int = 2, l_d: int = 22, n_layers: int = 32) -> float:
     return float(lib().oracle_cr_int(C.c_double(pi1), C.c_double(pi2), C.c_double(pi3), l_s, l_d, n_layers))
+
+
+# ------------------------------------------------------------------------------------------ O7 / O8 / cost model
+def merge_clusters(hidden: np.ndarray, vis_start: int, label: np.ndarray, keep_mask: np.ndarray):
+    """Eq. 6 on one sample: hidden bf16 bits [N, Dh], label / keep_mask [n].
+
+    Returns (merged float64 [M, Dh], merged_label int32 [M], merged_count int32 [M]), clusters in ascending label."""
+    h = _u16(hidden)
+    N, Dh = h.shape
+    lab = np.ascontiguousarray(label, dtype=np.int32)
+    keep = np.ascontiguousarray(keep_mask, dtype=np.uint8)
+    n = lab.shape[0]
+    cap = max(n, 1)
+    merged = np.zeros((cap, Dh), dtype=np.float64)
+    mlab = np.zeros(cap, dtype=np.int32)
+    mcnt = np.zeros(cap, dtype=np.int32)
+    m = lib().oracle_merge_clusters(_p(h), N, Dh, int(vis_start), n, _p(lab), _p(keep), _p(merged), _p(mlab), _p(mcnt),
+                                    cap)
+    return merged[:m].copy(), mlab[:m].copy(), mcnt[:m].copy()
+
+
+def cls_saliency(q_bits: np.ndarray, K_bits: np.ndarray, scale: float):
+    """Eq. 1 on one image: q bf16 bits [H, d], K [H, M, d] (key 0 = [CLS]) -> (S float64 [M-1], self-attention of [CLS])."""
+    q, K = _u16(q_bits), _u16(K_bits)
+    H, M, d = K.shape
+    S = np.zeros(max(M - 1, 0), dtype=np.float64)
+    c = C.c_double(0.0)
+    lib().oracle_cls_saliency(_p(q), _p(K), H, M, d, C.c_double(scale), _p(S), C.byref(c))
+    return S, float(c.value)
+
+
+def flops_layer(N: float, d: float) -> float:
+    return float(lib().oracle_flops_layer(C.c_double(N), C.c_double(d)))
+
+
+def visual_tokens_at_layer(l: int, m: float, pi1: float, pi2: float, pi3: float, l_s: int = 2, l_d: int = 22) -> float:
+    return float(lib().oracle_visual_tokens_at_layer(int(l), C.c_double(m), C.c_double(pi1), C.c_double(pi2),
+                                                     C.c_double(pi3), l_s, l_d))
+
+
+def flops_vitcop(m: float, n_text: float, d: float, pi1: float, pi2: float, pi3: float, l_s: int = 2, l_d: int = 22,
+                 n_layers: int = 32) -> float:
+    return float(lib().oracle_flops_vitcop(C.c_double(m), C.c_double(n_text), C.c_double(d), C.c_double(pi1),
+                                           C.c_double(pi2), C.c_double(pi3), l_s, l_d, n_layers))
 
 
 __all__ = [n for n in dir() if not n.startswith("_") and n not in ("C", "np", "os", "hashlib", "platform",

@@ -25,6 +25,10 @@
 //   R5  top-k ties go to the lower index; kept tokens are reported in ascending index order.
 //   R6  the quota of Eq. 5 is evaluated in exact integer arithmetic: q_c = (|C_c| * (B - N_c)) div n.
 //   R7  NaN scores sort after every number (they are pruned first when the smallest are kept).
+//   R8  merged rows (Eq. 6) come out in ascending order of their cluster label; where they are placed in the
+//       sequence is left to the caller (Algorithm 3 returns an unordered union).
+//   R9  the softmax of Eq. 1 runs over all keys of the layer, the [CLS] key included; scores are reported for
+//       the visual tokens only.
 
 #include <algorithm>
 #include <cmath>
@@ -359,6 +363,87 @@ int oracle_stage_count(int m, double pi) { return static_cast<int>(std::floor(st
 double oracle_cr_int(double pi1, double pi2, double pi3, int l_s, int l_d, int n_layers) {
     const double kept = pi1 * (l_s - 1) + pi2 * (l_d - l_s) + pi3 * (n_layers - l_d + 1);
     return 1.0 - kept / n_layers;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O7. Cluster merge, Eq. 6 / Algorithm 3 second half, for one sample: every cluster's tokens that were NOT
+//   kept as elites are averaged into one representative row,
+//       t_c^merged = (1 / |C_c^remaining|) * sum_{i in C_c^remaining} t_i .
+//   hidden [N, Dh] bf16 bits, the visual span starts at vis_start and has n tokens; label[n], keep[n] (1 = elite).
+//   Clusters are visited in ascending label value; a cluster without remaining tokens yields no row.
+//   merged [Mcap, Dh] doubles, merged_label / merged_count [Mcap]; returns the number of merged rows.
+//   (Where the merged rows go in the sequence is the caller's choice: Algorithm 3 returns a set.)
+// ---------------------------------------------------------------------------------------------
+int oracle_merge_clusters(const uint16_t* hidden, int N, int Dh, int vis_start, int n, const int32_t* label,
+                          const uint8_t* keep, double* merged, int32_t* merged_label, int32_t* merged_count,
+                          int Mcap) {
+    (void)N;
+    std::vector<int32_t> labs(label, label + n);
+    std::sort(labs.begin(), labs.end());
+    labs.erase(std::unique(labs.begin(), labs.end()), labs.end());
+    int m = 0;
+    for (int32_t lab : labs) {
+        std::vector<int> rest;
+        for (int i = 0; i < n; ++i)
+            if (label[i] == lab && !keep[i]) rest.push_back(i);
+        if (rest.empty()) continue;
+        if (m < Mcap) {
+            for (int e = 0; e < Dh; ++e) {
+                double acc = 0.0;
+                for (int i : rest) acc += bf16_to_double(hidden[static_cast<size_t>(vis_start + i) * Dh + e]);
+                merged[static_cast<size_t>(m) * Dh + e] = acc / static_cast<double>(rest.size());
+            }
+            merged_label[m] = lab;
+            merged_count[m] = static_cast<int32_t>(rest.size());
+        }
+        ++m;
+    }
+    return m;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O8. Stage I saliency, Eq. 1, for one image:  S_i = sum_h A^(h)_{0,i}, where A^(h) is the attention matrix
+//   of head h of the vision encoder layer and row 0 belongs to the [CLS] token:
+//       A^(h)_{0,j} = softmax_j( scale * q^(h) . k_j^(h) ),   j = 0 .. M-1   (key 0 is [CLS] itself).
+//   q [H, d] is the [CLS] query, K [H, M, d] the keys (bf16 bits).  S [M-1] receives the scores of the visual
+//   tokens j = 1 .. M-1; cls_out (optional) the attention [CLS] pays to itself, summed over heads.
+// ---------------------------------------------------------------------------------------------
+void oracle_cls_saliency(const uint16_t* q, const uint16_t* K, int H, int M, int d, double scale, double* S,
+                         double* cls_out) {
+    std::vector<double> total(M, 0.0), logit(M);
+    for (int h = 0; h < H; ++h) {
+        double mx = -std::numeric_limits<double>::infinity();
+        for (int j = 0; j < M; ++j) {
+            double acc = 0.0;
+            for (int e = 0; e < d; ++e)
+                acc += bf16_to_double(q[static_cast<size_t>(h) * d + e]) *
+                       bf16_to_double(K[(static_cast<size_t>(h) * M + j) * d + e]);
+            logit[j] = scale * acc;
+            mx = std::max(mx, logit[j]);
+        }
+        double den = 0.0;
+        for (int j = 0; j < M; ++j) den += std::exp(logit[j] - mx);
+        for (int j = 0; j < M; ++j) total[j] += std::exp(logit[j] - mx) / den;
+    }
+    for (int j = 1; j < M; ++j) S[j - 1] = total[j];
+    if (cls_out) *cls_out = total[0];
+}
+
+// Cost model of Appendix E.  Eq. 7: FLOPs of one transformer layer on a sequence of N tokens, hidden size d.
+double oracle_flops_layer(double N, double d) { return 4.0 * N * N * d + 16.0 * N * d * d; }
+
+// Eq. 8: visual tokens present at layer l (1-based) of an n-layer LLM: pi1*m before l_s, pi2*m from l_s, pi3*m from l_d.
+double oracle_visual_tokens_at_layer(int l, double m, double pi1, double pi2, double pi3, int l_s, int l_d) {
+    if (l < l_s) return pi1 * m;
+    if (l < l_d) return pi2 * m;
+    return pi3 * m;
+}
+
+// Eq. 9: total FLOPs of the LLM with the three-stage schedule (N_t text tokens ride along at every layer).
+double oracle_flops_vitcop(double m, double n_text, double d, double pi1, double pi2, double pi3, int l_s, int l_d,
+                           int n_layers) {
+    return (l_s - 1) * oracle_flops_layer(pi1 * m + n_text, d) + (l_d - l_s) * oracle_flops_layer(pi2 * m + n_text, d) +
+           (n_layers - l_d + 1) * oracle_flops_layer(pi3 * m + n_text, d);
 }
 
 }  // extern "C"

@@ -499,3 +499,93 @@ def test_chain_kept_count_equals_budget():
             keep = oracle.select_plain(s[b], k)
             assert len(keep) == min(k, n)
         n = min(k, n)
+
+
+# ======================================================================================= Eq. 6: cluster merge
+def test_merge_hand_example():
+    # four tokens, Dh = 2, labels {0,0,2,2}, token 0 kept: cluster 0 averages token 1 alone, cluster 2 averages 2 and 3
+    hid = W.f32_to_bf16_bits(np.array([[9, 9], [1, 2], [3, 5], [4, 6], [5, 7]], dtype=np.float32))   # row 0 is text
+    merged, mlab, mcnt = oracle.merge_clusters(hid, 1, np.array([0, 0, 2, 2]), np.array([1, 0, 0, 0]))
+    assert mlab.tolist() == [0, 2] and mcnt.tolist() == [1, 2]
+    assert np.array_equal(merged, np.array([[3.0, 5.0], [4.5, 6.5]]))
+    # every token of a cluster kept -> no merged row for it
+    merged, mlab, mcnt = oracle.merge_clusters(hid, 1, np.array([0, 0, 2, 2]), np.array([1, 1, 0, 1]))
+    assert mlab.tolist() == [2] and mcnt.tolist() == [1] and np.array_equal(merged, np.array([[4.0, 6.0]]))
+
+
+def test_merge_conservation_and_library_mean():
+    rng = np.random.default_rng(5)
+    n, Dh, vs = 97, 24, 3
+    hid = W.f32_to_bf16_bits(rng.standard_normal((vs + n + 2, Dh)).astype(np.float32))
+    x = W.bf16_bits_to_f32(hid).astype(np.float64)[vs:vs + n]
+    label = W.make_labels(3, 1, n, 7)[0]
+    keep = (rng.random(n) < 0.3).astype(np.uint8)
+    merged, mlab, mcnt = oracle.merge_clusters(hid, vs, label, keep)
+    # counts: every non-elite token is averaged exactly once
+    assert mcnt.sum() == n - keep.sum() and np.all(np.diff(mlab) > 0)
+    # conservation: sum_c count_c * merged_c + sum of elite rows == sum of all rows
+    assert np.allclose((merged * mcnt[:, None]).sum(0) + x[keep == 1].sum(0), x.sum(0), rtol=0, atol=1e-10)
+    # each row against numpy's mean over the members
+    for r, lab in enumerate(mlab):
+        members = (label == lab) & (keep == 0)
+        assert np.allclose(merged[r], x[members].mean(0), rtol=0, atol=1e-13)
+    # a single cluster with nothing kept is the plain column mean; constant rows average to the constant
+    merged, _, mcnt = oracle.merge_clusters(hid, vs, np.zeros(n, np.int32), np.zeros(n, np.uint8))
+    assert mcnt.tolist() == [n] and np.allclose(merged[0], x.mean(0), atol=1e-13)
+    const = W.f32_to_bf16_bits(np.full((n, Dh), 1.5, dtype=np.float32))
+    merged, _, _ = oracle.merge_clusters(const, 0, label, keep)
+    assert np.all(merged == 1.5)
+
+
+# ======================================================================================= Eq. 1: [CLS] saliency
+def test_cls_saliency_closed_forms():
+    H, M, d = 4, 33, 16
+    rng = np.random.default_rng(2)
+    q = W.f32_to_bf16_bits(rng.standard_normal((H, d)).astype(np.float32))
+    # identical keys: every attention row is uniform, S_i = H / M
+    K = np.tile(W.f32_to_bf16_bits(rng.standard_normal((H, 1, d)).astype(np.float32)), (1, M, 1))
+    S, c = oracle.cls_saliency(q, K, 0.25)
+    assert np.allclose(S, H / M, atol=1e-14) and abs(c - H / M) < 1e-14
+    # each head's row sums to one: [CLS] share + visual shares == H
+    K = W.f32_to_bf16_bits(rng.standard_normal((H, M, d)).astype(np.float32))
+    S, c = oracle.cls_saliency(q, K, 0.25)
+    assert abs(S.sum() + c - H) < 1e-12 and np.all(S > 0)
+    # against a library softmax on the same logits
+    from scipy.special import softmax
+    qf, Kf = W.bf16_bits_to_f32(q).astype(np.float64), W.bf16_bits_to_f32(K).astype(np.float64)
+    ref = softmax(0.25 * np.einsum("hd,hmd->hm", qf, Kf), axis=1).sum(0)
+    assert np.allclose(S, ref[1:], rtol=1e-12, atol=0)
+    # shifting every key by one vector adds the same constant to all logits of a head: S unchanged
+    shift = W.bf16_bits_to_f32(W.f32_to_bf16_bits(np.full((1, 1, d), 0.5, dtype=np.float32)))
+    K2 = W.f32_to_bf16_bits((W.bf16_bits_to_f32(K) * 0.5).astype(np.float32))       # exact halving keeps bf16 exact
+    K3 = W.f32_to_bf16_bits((W.bf16_bits_to_f32(K2) + shift).astype(np.float32))
+    exact = np.array_equal(W.bf16_bits_to_f32(K3), W.bf16_bits_to_f32(K2) + shift)
+    S2, _ = oracle.cls_saliency(q, K2, 0.25)
+    S3, _ = oracle.cls_saliency(q, K3, 0.25)
+    if exact:
+        assert np.allclose(S2, S3, rtol=1e-10)
+    # one key aligned with the query and a large scale: that token takes (almost) all the attention of every head
+    K = np.zeros((H, M, d), dtype=np.float32)
+    K[:, 7] = W.bf16_bits_to_f32(q)
+    S, c = oracle.cls_saliency(q, W.f32_to_bf16_bits(K), 50.0)
+    assert abs(S[6] - H) < 1e-6 and S[6] == S.max()
+
+
+# ======================================================================================= Eq. 7-9: cost model
+def test_cost_model_closed_forms():
+    assert oracle.flops_layer(1, 1) == 20.0
+    assert oracle.flops_layer(3, 2) == 4 * 9 * 2 + 16 * 3 * 4
+    # Eq. 8 boundaries with l_s = 2, l_d = 22
+    m, p = 576.0, (0.5, 0.4394, 0.0879)
+    assert oracle.visual_tokens_at_layer(1, m, *p) == 0.5 * m
+    assert oracle.visual_tokens_at_layer(2, m, *p) == 0.4394 * m == oracle.visual_tokens_at_layer(21, m, *p)
+    assert oracle.visual_tokens_at_layer(22, m, *p) == 0.0879 * m == oracle.visual_tokens_at_layer(32, m, *p)
+    # Eq. 9 is the sum of Eq. 7 over the layers with the token count of Eq. 8
+    tot = sum(oracle.flops_layer(oracle.visual_tokens_at_layer(l, m, *p) + 64, 4096) for l in range(1, 33))
+    assert abs(oracle.flops_vitcop(m, 64, 4096, *p) - tot) <= 1e-9 * tot
+    # no pruning: n layers at full length; Eq. 10 is then zero
+    assert oracle.flops_vitcop(m, 64, 4096, 1, 1, 1) == 32 * oracle.flops_layer(m + 64, 4096)
+    assert oracle.cr_int(1, 1, 1) == 0.0
+    # Eq. 10 equals one minus the layer average of Eq. 8 over m
+    avg = sum(oracle.visual_tokens_at_layer(l, m, *p) for l in range(1, 33)) / (32 * m)
+    assert abs(oracle.cr_int(*p) - (1 - avg)) < 1e-15
