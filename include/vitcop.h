@@ -50,6 +50,7 @@ extern "C" {
 #define VITCOP_OP_COMPACT     3
 #define VITCOP_OP_PRUNE_STEP  4
 #define VITCOP_OP_SIMILARITY  5
+#define VITCOP_OP_SALIENCY    6   /* vitcop_cls_saliency: B = images, H = heads, N = keys per head (M) */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* vitcop_status_string(int status);
@@ -214,6 +215,58 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V,
                       int32_t* kept_pos, int32_t* out_len,
                       float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- cluster merge
+ * Eq. 6 of the paper (second half of Algorithm 3): in every cluster the tokens that were NOT kept as elites are
+ * averaged into one representative token, t_c = (1 / |R_c|) * sum_{i in R_c} t_i, so that a pruning step returns
+ * the elites plus one merged token per cluster.  Rows are summed in fp32 in ascending token order.
+ * Readings where the paper is silent: the merged tokens are hidden-state rows; they come out as a separate
+ * tensor, one row per cluster that has non-elite tokens, in ascending order of the cluster's label (Algorithm 3
+ * returns an unordered union, so where they go in the sequence is the caller's choice); a cluster whose tokens
+ * were all kept yields no row.
+ *   hidden        bf16 [B, N, Dh]   (Dh multiple of 8)
+ *   label         int32 [B, Nv_cap]  cluster labels of the span, as written by vitcop_redundancy_filter
+ *   keep_mask     uint8 [B, Nv_cap]  1 = elite (kept), as written by vitcop_select
+ *   merged        bf16 [B, Mcap, Dh] out, optional: the averages rounded to nearest even
+ *   merged_f32    fp32 [B, Mcap, Dh] out, optional: the averages before that rounding
+ *   merged_label  int32 [B, Mcap] out: label of each merged row;  merged_count int32 [B, Mcap] out: |R_c|
+ *   n_merged      int32 [B] out: number of clusters with non-elite tokens (rows past Mcap are not written)
+ * Errors: INVALID_ARG, UNSUPPORTED (Dh % 8, alignment, Nv_cap > VITCOP_MAX_VISUAL_TOKENS), CUDA. */
+int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh,
+                          int vis_start, const int32_t* vis_len, int vis_len_uniform, int Nv_cap,
+                          const int32_t* label, const uint8_t* keep_mask,
+                          void* merged, float* merged_f32, int32_t* merged_label, int32_t* merged_count,
+                          int32_t* n_merged, int Mcap, void* stream);
+
+/* ---------------------------------------------------------------- Stage I saliency
+ * Eq. 1 of the paper: S_i = sum_h A^(h)_{0,i}, the attention that the [CLS] token (index 0) of the vision
+ * encoder pays to visual token i, summed over the heads; Stage I keeps the tokens with the LARGEST S
+ * (vitcop_select with largest = 1, then vitcop_compact_kv on the feature rows).
+ * A^(h)_{0,j} = softmax over all M keys j (the [CLS] key included) of scale * q^(h) . k_j^(h).
+ *   q_cls     bf16 [B, H, d]      query of the [CLS] token per head (d multiple of 8)
+ *   K         bf16 [B, H, M, d]   keys of the layer; key 0 belongs to [CLS]
+ *   scale     usually 1 / sqrt(d)
+ *   saliency  fp32 [B, M - 1] out: S of the visual tokens 1 .. M-1
+ *   cls_self  fp32 [B] out, optional: attention of [CLS] to itself, summed over heads
+ *   workspace vitcop_workspace_bytes(VITCOP_OP_SALIENCY, B, H, M, ...) bytes
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, int d, float scale,
+                        float* saliency, float* cls_self, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- schedule and cost model (host arithmetic)
+ * Algorithm 1 prunes to floor(m * pi) tokens per stage (pi relative to the ORIGINAL m visual tokens); Appendix E
+ * models the cost.  Layers are numbered from 1; Stage II acts at layer l_s, Stage III at layer l_d.
+ *   vitcop_stage_count            floor(m * pi), evaluated in double
+ *   vitcop_flops_layer            Eq. 7: 4 N^2 d + 16 N d^2
+ *   vitcop_visual_tokens_at_layer Eq. 8: pi1*m for l < l_s, pi2*m for l_s <= l < l_d, pi3*m from l_d on
+ *   vitcop_flops_total            Eq. 9: sum over the n_layers layers of Eq. 7 at Eq. 8's length plus n_text
+ *   vitcop_cr_int                 Eq. 10: one minus the layer average of Eq. 8 over m */
+int    vitcop_stage_count(int m, double pi);
+double vitcop_flops_layer(double N, double d);
+double vitcop_visual_tokens_at_layer(int l, double m, double pi1, double pi2, double pi3, int l_s, int l_d);
+double vitcop_flops_total(double m, double n_text, double d, double pi1, double pi2, double pi3,
+                          int l_s, int l_d, int n_layers);
+double vitcop_cr_int(double pi1, double pi2, double pi3, int l_s, int l_d, int n_layers);
 
 /* ---------------------------------------------------------------- fused pruning step without a workspace
  * The paper has no counterpart: this is vitcop_prune_step for callers that have no way to obtain device

@@ -18,14 +18,15 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvitcop.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT = range(7)
-OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY = range(6)
+OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY = range(7)
 MAX_VISUAL_TOKENS = 16384
 
 EXPORTS = [
     "vitcop_status_string", "vitcop_last_cuda_error", "vitcop_workspace_bytes", "vitcop_poll_status",
     "vitcop_redundancy_filter", "vitcop_similarity_rows", "vitcop_knorm_score", "vitcop_select",
     "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
-    "vitcop_prune_step_static",
+    "vitcop_prune_step_static", "vitcop_merge_clusters", "vitcop_cls_saliency", "vitcop_stage_count",
+    "vitcop_flops_layer", "vitcop_visual_tokens_at_layer", "vitcop_flops_total", "vitcop_cr_int",
 ]
 
 
@@ -78,6 +79,18 @@ def lib() -> C.CDLL:
                                         vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.vitcop_prune_step_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, vp, i32, i32, vp, i32,
                                                vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+        L.vitcop_merge_clusters.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp]
+        L.vitcop_cls_saliency.argtypes = [vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp, sz, vp]
+        f64 = C.c_double
+        L.vitcop_stage_count.argtypes = [i32, f64]
+        L.vitcop_flops_layer.argtypes = [f64, f64]
+        L.vitcop_flops_layer.restype = f64
+        L.vitcop_visual_tokens_at_layer.argtypes = [i32, f64, f64, f64, f64, i32, i32]
+        L.vitcop_visual_tokens_at_layer.restype = f64
+        L.vitcop_flops_total.argtypes = [f64, f64, f64, f64, f64, f64, i32, i32, i32]
+        L.vitcop_flops_total.restype = f64
+        L.vitcop_cr_int.argtypes = [f64, f64, f64, i32, i32, i32]
+        L.vitcop_cr_int.restype = f64
         L.vitcop_kernel_timing_begin.argtypes = []
         L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
@@ -209,6 +222,52 @@ def vitcop_prune_step_static(hidden, K, V, vis_start: int, vis_len, Nv_cap: int,
                                         _ptr(keep_idx_out), _ptr(n_keep_out), _stream())
     _check(rc, "vitcop_prune_step_static")
     return out_len
+
+
+def vitcop_merge_clusters(hidden, vis_start: int, vis_len, label, keep_mask, merged_label, merged_count, n_merged,
+                          merged=None, merged_f32=None):
+    """Eq. 6: one averaged row per cluster that has non-elite tokens (``keep_mask`` 0), ascending label order."""
+    B, N, Dh = hidden.shape
+    Nv_cap = label.shape[1]
+    Mcap = merged_label.shape[1]
+    vp, vu = _vis(vis_len)
+    rc = lib().vitcop_merge_clusters(_ptr(hidden), B, N, Dh, vis_start, vp, vu, Nv_cap, _ptr(label), _ptr(keep_mask),
+                                     _ptr(merged), _ptr(merged_f32), _ptr(merged_label), _ptr(merged_count),
+                                     _ptr(n_merged), Mcap, _stream())
+    _check(rc, "vitcop_merge_clusters")
+    return n_merged
+
+
+def vitcop_cls_saliency(q_cls, K, scale: float, saliency, workspace, cls_self=None):
+    """Eq. 1: q_cls bf16 [B,H,d], K bf16 [B,H,M,d] (key 0 = [CLS]) -> saliency fp32 [B, M-1]."""
+    B, H, M, d = K.shape
+    rc = lib().vitcop_cls_saliency(_ptr(q_cls), _ptr(K), B, H, M, d, float(scale), _ptr(saliency), _ptr(cls_self),
+                                   _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "vitcop_cls_saliency")
+    return saliency
+
+
+def vitcop_stage_count(m: int, pi: float) -> int:
+    return int(lib().vitcop_stage_count(int(m), float(pi)))
+
+
+def vitcop_flops_layer(N: float, d: float) -> float:
+    return float(lib().vitcop_flops_layer(float(N), float(d)))
+
+
+def vitcop_visual_tokens_at_layer(l: int, m: float, pi1: float, pi2: float, pi3: float, l_s: int = 2,
+                                  l_d: int = 22) -> float:
+    return float(lib().vitcop_visual_tokens_at_layer(int(l), float(m), float(pi1), float(pi2), float(pi3), l_s, l_d))
+
+
+def vitcop_flops_total(m: float, n_text: float, d: float, pi1: float, pi2: float, pi3: float, l_s: int = 2,
+                       l_d: int = 22, n_layers: int = 32) -> float:
+    return float(lib().vitcop_flops_total(float(m), float(n_text), float(d), float(pi1), float(pi2), float(pi3), l_s,
+                                          l_d, n_layers))
+
+
+def vitcop_cr_int(pi1: float, pi2: float, pi3: float, l_s: int = 2, l_d: int = 22, n_layers: int = 32) -> float:
+    return float(lib().vitcop_cr_int(float(pi1), float(pi2), float(pi3), l_s, l_d, n_layers))
 
 
 def vitcop_redundancy_filter(feat: torch.Tensor, pos: Optional[torch.Tensor], label: torch.Tensor,

@@ -180,7 +180,7 @@ int vitcop_kernel_timing_end(vitcop_kernel_time* out, int capacity, int* count) 
 }
 
 int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, int Dh, size_t* bytes) {
-    (void)H; (void)N; (void)d; (void)Dh;
+    (void)d; (void)Dh;
     if (!bytes || B < 0 || Nv < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
     switch (op) {
         case VITCOP_OP_FILTER: *bytes = filter_workspace_bytes(B, Nv, D); return VITCOP_OK;
@@ -189,6 +189,10 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
         case VITCOP_OP_COMPACT: *bytes = 0; return VITCOP_OK;
         case VITCOP_OP_SELECT: *bytes = kStatusBytes; return VITCOP_OK;
         case VITCOP_OP_PRUNE_STEP: *bytes = StepWs(B, Nv).total; return VITCOP_OK;
+        case VITCOP_OP_SALIENCY:
+            if (H < 0 || N < 0) return VITCOP_ERR_INVALID_ARG;
+            *bytes = saliency_workspace_bytes(B, H, N);
+            return VITCOP_OK;
         default: return VITCOP_ERR_INVALID_ARG;
     }
 }
@@ -305,6 +309,33 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, i
     if (rc != VITCOP_OK) return rc;
     return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep, Nv_cap,
                           nkeep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, s, true);
+}
+
+int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh, int vis_start, const int32_t* vis_len,
+                          int vis_len_uniform, int Nv_cap, const int32_t* label, const uint8_t* keep_mask, void* merged,
+                          float* merged_f32, int32_t* merged_label, int32_t* merged_count, int32_t* n_merged, int Mcap,
+                          void* stream) {
+    if (!hidden || !label || !keep_mask || !merged_label || !merged_count || !n_merged) return VITCOP_ERR_INVALID_ARG;
+    if (B < 0 || N < 0 || Dh < 0 || Nv_cap < 0 || Mcap < 0) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_span(N, vis_start, vis_len, vis_len_uniform, Nv_cap);
+    if (rc != VITCOP_OK) return rc;
+    if (Dh % 8 || !aligned16(hidden) || !aligned16(merged) || !aligned16(merged_f32)) return VITCOP_ERR_UNSUPPORTED;
+    if (Nv_cap > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    return launch_merge(hidden, B, N, Dh, vis_start, vis_len, vis_len_uniform, Nv_cap, label, keep_mask, merged,
+                        merged_f32, merged_label, merged_count, n_merged, Mcap, static_cast<cudaStream_t>(stream));
+}
+
+int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, int d, float scale, float* saliency,
+                        float* cls_self, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!q_cls || !K || !saliency || B < 0 || H < 0 || M < 0 || d < 0) return VITCOP_ERR_INVALID_ARG;
+    if (d % 8 || !aligned16(q_cls) || !aligned16(K) || B > 65535 || d > 4096) return VITCOP_ERR_UNSUPPORTED;
+    if ((size_t)(d + M) * sizeof(float) > 200 * 1024) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < saliency_workspace_bytes(B, H, M) || !aligned256(workspace))
+        return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    return launch_cls_saliency(q_cls, K, B, H, M, d, scale, saliency, cls_self, workspace, s);
 }
 
 int vitcop_prune_step_static(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,

@@ -21,7 +21,7 @@ import numpy as np
 
 __all__ = [
     "Workload", "WORKLOADS", "workload", "f32_to_bf16_bits", "bf16_bits_to_f32",
-    "make_features", "make_positions", "make_kv", "make_hidden", "make_scores", "make_labels",
+    "make_features", "make_positions", "make_kv", "make_hidden", "make_scores", "make_labels", "make_cls_qk",
 ]
 
 
@@ -271,3 +271,20 @@ def make_labels(seed: int, B: int, n: int, n_clusters: int) -> np.ndarray:
         lab[centres] = centres                                  # a centre carries its own index
         out[b] = lab
     return out
+
+
+def make_cls_qk(seed: int, B: int, H: int, M: int, d: int, salient: float = 0.05) -> Tuple[np.ndarray, np.ndarray]:
+    """bf16 bits q [B, H, d] and K [B, H, M, d] of one vision-encoder layer (key 0 belongs to [CLS]).
+
+    Keys are N(0,1); a fraction ``salient`` of the tokens gets a component along the head's query, so that the
+    [CLS] attention row is peaked on a few tokens the way a trained encoder's is (shapes of CLIP ViT-L/14-336:
+    H = 16, d = 64, M = 577)."""
+    rng = _rng(seed, 33, 9, M)
+    q = rng.standard_normal((B, H, d), dtype=np.float32)
+    K = rng.standard_normal((B, H, M, d), dtype=np.float32)
+    n_sal = max(1, int(salient * M))
+    for b in range(B):
+        idx = rng.permutation(M)[:n_sal]
+        gain = rng.uniform(0.5, 1.5, size=n_sal).astype(np.float32)
+        K[b, :, idx] += (gain[:, None, None] * q[b][None, :, :]).astype(np.float32)
+    return f32_to_bf16_bits(q), f32_to_bf16_bits(K)
