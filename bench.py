@@ -381,10 +381,30 @@ def run_ours(args):
                                                 st.Ko, st.Vo, st.olen, kept_pos=st.kpos),
         "prune_step": st.prune,
     }
+    # the two stages around the core chain: cluster merge (Eq. 6) after the step, Stage I saliency (Eq. 1) before it
+    kmask = torch.empty((w.B, w.Nv), dtype=torch.uint8, device=dev)
+    vb.vitcop_select(score, w.Nv, st.budget, kidx, st.nkeep, ws_sel, label=st.label, keep_mask=kmask)
+    m_lab = torch.empty((w.B, w.n_centers), dtype=torch.int32, device=dev)
+    m_cnt, n_mrg = torch.empty_like(m_lab), torch.empty((w.B,), dtype=torch.int32, device=dev)
+    m_rows = torch.empty((w.B, w.n_centers, w.Dh), dtype=torch.bfloat16, device=dev)
+    vit_H, vit_M, vit_d = 16, 577, 64                   # CLIP ViT-L/14-336: 16 heads of 64, [CLS] + 576 patches
+    q_b, Kv_b = W.make_cls_qk(w.seed, w.B, vit_H, vit_M, vit_d)
+    q_cls, K_vit = vb.bf16_tensor(q_b, dev), vb.bf16_tensor(Kv_b, dev)
+    sal = torch.empty((w.B, vit_M - 1), dtype=torch.float32, device=dev)
+    ws_sal = vb.alloc_workspace(vb.OP_SALIENCY, device=dev, B=w.B, H=vit_H, N=vit_M)
+    ws_mrg = vb.alloc_workspace(vb.OP_MERGE, device=dev, B=w.B, Nv=w.Nv, N=w.n_centers)
+    stage_fns["merge"] = lambda: vb.vitcop_merge_clusters(st.hidden, w.vis_start, w.Nv, st.label, kmask, m_lab, m_cnt,
+                                                          n_mrg, ws_mrg, merged=m_rows)
+    stage_fns["cls_saliency"] = lambda: vb.vitcop_cls_saliency(q_cls, K_vit, vit_d ** -0.5, sal, ws_sal)
     stage = {}
     for name, fn in stage_fns.items():
         t = timed(fn, n_kt, 3)
         stage[name] = {"us_median": float(np.median(t) * 1e3), "us_min": float(t.min() * 1e3)}
+    merged_rows = int(m_cnt.cpu().numpy()[np.arange(w.n_centers)[None, :] < n_mrg.cpu().numpy()[:, None]].sum())
+    for name, nbytes in (("merge", (merged_rows + int(n_mrg.sum())) * w.Dh * 2 + w.B * w.Nv * 5),
+                         ("cls_saliency", w.B * vit_H * vit_M * vit_d * 2 + w.B * vit_H * vit_M * 8)):
+        gbs = nbytes / (stage[name]["us_median"] * 1e-6) / 1e9
+        stage[name].update(algorithmic_bytes=nbytes, gbs=gbs, frac_of_measured_hbm=gbs / peaks["hbm_gbs"])
 
     # end to end through the public API with host buffers ----------------------------------------------------
     out_host = {"ho": torch.empty(st.ho.shape, dtype=st.ho.dtype).pin_memory(),

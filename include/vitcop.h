@@ -51,6 +51,7 @@ extern "C" {
 #define VITCOP_OP_PRUNE_STEP  4
 #define VITCOP_OP_SIMILARITY  5
 #define VITCOP_OP_SALIENCY    6   /* vitcop_cls_saliency: B = images, H = heads, N = keys per head (M) */
+#define VITCOP_OP_MERGE       7   /* vitcop_merge_clusters: Nv = Nv_cap, N = Mcap */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* vitcop_status_string(int status);
@@ -231,12 +232,13 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V,
  *   merged_f32    fp32 [B, Mcap, Dh] out, optional: the averages before that rounding
  *   merged_label  int32 [B, Mcap] out: label of each merged row;  merged_count int32 [B, Mcap] out: |R_c|
  *   n_merged      int32 [B] out: number of clusters with non-elite tokens (rows past Mcap are not written)
- * Errors: INVALID_ARG, UNSUPPORTED (Dh % 8, alignment, Nv_cap > VITCOP_MAX_VISUAL_TOKENS), CUDA. */
+ *   workspace     vitcop_workspace_bytes(VITCOP_OP_MERGE, B, 0, Mcap, 0, Nv_cap, 0, 0) bytes
+ * Errors: INVALID_ARG, UNSUPPORTED (Dh % 8, alignment, Nv_cap > VITCOP_MAX_VISUAL_TOKENS), WORKSPACE, CUDA. */
 int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh,
                           int vis_start, const int32_t* vis_len, int vis_len_uniform, int Nv_cap,
                           const int32_t* label, const uint8_t* keep_mask,
                           void* merged, float* merged_f32, int32_t* merged_label, int32_t* merged_count,
-                          int32_t* n_merged, int Mcap, void* stream);
+                          int32_t* n_merged, int Mcap, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------- Stage I saliency
  * Eq. 1 of the paper: S_i = sum_h A^(h)_{0,i}, the attention that the [CLS] token (index 0) of the vision

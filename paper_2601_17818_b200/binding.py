@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvitcop.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT = range(7)
-OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY = range(7)
+OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY, OP_MERGE = range(8)
 MAX_VISUAL_TOKENS = 16384
 
 EXPORTS = [
@@ -79,7 +79,8 @@ def lib() -> C.CDLL:
                                         vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.vitcop_prune_step_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, vp, i32, i32, vp, i32,
                                                vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
-        L.vitcop_merge_clusters.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp]
+        L.vitcop_merge_clusters.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz,
+                                            vp]
         L.vitcop_cls_saliency.argtypes = [vp, vp, i32, i32, i32, i32, C.c_float, vp, vp, vp, sz, vp]
         f64 = C.c_double
         L.vitcop_stage_count.argtypes = [i32, f64]
@@ -225,7 +226,7 @@ def vitcop_prune_step_static(hidden, K, V, vis_start: int, vis_len, Nv_cap: int,
 
 
 def vitcop_merge_clusters(hidden, vis_start: int, vis_len, label, keep_mask, merged_label, merged_count, n_merged,
-                          merged=None, merged_f32=None):
+                          workspace, merged=None, merged_f32=None):
     """Eq. 6: one averaged row per cluster that has non-elite tokens (``keep_mask`` 0), ascending label order."""
     B, N, Dh = hidden.shape
     Nv_cap = label.shape[1]
@@ -233,7 +234,7 @@ def vitcop_merge_clusters(hidden, vis_start: int, vis_len, label, keep_mask, mer
     vp, vu = _vis(vis_len)
     rc = lib().vitcop_merge_clusters(_ptr(hidden), B, N, Dh, vis_start, vp, vu, Nv_cap, _ptr(label), _ptr(keep_mask),
                                      _ptr(merged), _ptr(merged_f32), _ptr(merged_label), _ptr(merged_count),
-                                     _ptr(n_merged), Mcap, _stream())
+                                     _ptr(n_merged), Mcap, _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "vitcop_merge_clusters")
     return n_merged
 

@@ -189,6 +189,10 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
         case VITCOP_OP_COMPACT: *bytes = 0; return VITCOP_OK;
         case VITCOP_OP_SELECT: *bytes = kStatusBytes; return VITCOP_OK;
         case VITCOP_OP_PRUNE_STEP: *bytes = StepWs(B, Nv).total; return VITCOP_OK;
+        case VITCOP_OP_MERGE:
+            if (N < 0) return VITCOP_ERR_INVALID_ARG;
+            *bytes = merge_workspace_bytes(B, Nv, N);
+            return VITCOP_OK;
         case VITCOP_OP_SALIENCY:
             if (H < 0 || N < 0) return VITCOP_ERR_INVALID_ARG;
             *bytes = saliency_workspace_bytes(B, H, N);
@@ -314,15 +318,20 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, i
 int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh, int vis_start, const int32_t* vis_len,
                           int vis_len_uniform, int Nv_cap, const int32_t* label, const uint8_t* keep_mask, void* merged,
                           float* merged_f32, int32_t* merged_label, int32_t* merged_count, int32_t* n_merged, int Mcap,
-                          void* stream) {
+                          void* workspace, size_t workspace_bytes, void* stream) {
     if (!hidden || !label || !keep_mask || !merged_label || !merged_count || !n_merged) return VITCOP_ERR_INVALID_ARG;
     if (B < 0 || N < 0 || Dh < 0 || Nv_cap < 0 || Mcap < 0) return VITCOP_ERR_INVALID_ARG;
     int rc = check_span(N, vis_start, vis_len, vis_len_uniform, Nv_cap);
     if (rc != VITCOP_OK) return rc;
     if (Dh % 8 || !aligned16(hidden) || !aligned16(merged) || !aligned16(merged_f32)) return VITCOP_ERR_UNSUPPORTED;
     if (Nv_cap > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < merge_workspace_bytes(B, Nv_cap, Mcap) || !aligned256(workspace))
+        return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
     return launch_merge(hidden, B, N, Dh, vis_start, vis_len, vis_len_uniform, Nv_cap, label, keep_mask, merged,
-                        merged_f32, merged_label, merged_count, n_merged, Mcap, static_cast<cudaStream_t>(stream));
+                        merged_f32, merged_label, merged_count, n_merged, Mcap, workspace, s);
 }
 
 int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, int d, float scale, float* saliency,

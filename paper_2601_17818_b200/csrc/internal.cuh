@@ -55,7 +55,9 @@ int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, in
 
 int launch_merge(const void* hidden, int B, int N, int Dh, int vis_start, const int32_t* vis_len, int vis_len_uniform,
                  int Nv_cap, const int32_t* label, const uint8_t* keep_mask, void* merged_bf16, float* merged_f32,
-                 int32_t* merged_label, int32_t* merged_count, int32_t* n_merged, int Mcap, cudaStream_t stream);
+                 int32_t* merged_label, int32_t* merged_count, int32_t* n_merged, int Mcap, void* workspace,
+                 cudaStream_t stream);
+size_t merge_workspace_bytes(int B, int Nv_cap, int Mcap);
 
 size_t saliency_workspace_bytes(int B, int H, int M);
 int launch_cls_saliency(const void* q, const void* K, int B, int H, int M, int d, float scale, float* saliency,

@@ -27,7 +27,8 @@ def _gpu_merge(hid_bits, vis_start, vis_len, label, keep_mask, Mcap):
     mc = torch.full((B, Mcap), -7, dtype=torch.int32, device=DEV)
     nm = torch.full((B,), -7, dtype=torch.int32, device=DEV)
     vl = int(vis_len) if np.isscalar(vis_len) else dev_i32(vis_len)
-    vb.vitcop_merge_clusters(hid, vis_start, vl, lab, km, ml, mc, nm, merged=mb, merged_f32=mf)
+    ws = vb.alloc_workspace(vb.OP_MERGE, B=B, Nv=lab.shape[1], N=Mcap)
+    vb.vitcop_merge_clusters(hid, vis_start, vl, lab, km, ml, mc, nm, ws, merged=mb, merged_f32=mf)
     torch.cuda.synchronize()
     return vb.bf16_bits(mb), mf.cpu().numpy(), ml.cpu().numpy(), mc.cpu().numpy(), nm.cpu().numpy()
 
