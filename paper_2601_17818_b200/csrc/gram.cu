@@ -245,6 +245,253 @@ struct GemmSmem {
 constexpr float kInf = __builtin_huge_valf();
 
 // ------------------------------------------------------------------------------------------------
+// epilogue of one output tile (called by all epilogue threads of the CTA)
+// ------------------------------------------------------------------------------------------------
+struct EpiSmem {
+    float *colw, *cola, *colrho, *colx, *coly, *colred, *rowred;
+    int *colidx, *rowidx;
+};
+struct EpiCall {
+    int b, ti, tj;                 // sample, row tile, column tile
+    uint32_t tmem_tile;            // TMEM address (lane 0) of the tile's first accumulator column
+    uint32_t wait_bar, wait_parity;   // mbarrier that completes when the accumulator is ready (0: it already is)
+    uint32_t arrive_bar;           // mbarrier to arrive on once this thread has read the accumulator (0: none)
+    volatile int* abort_flag;
+};
+
+// Returns true when the CTA must give up (a bounded wait expired somewhere).
+template <int BN, int MODE, int METRIC, bool SPATIAL, int NS>
+__device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm, const EpiCall& call, bool& ok) {
+    constexpr bool SYM = MODE == GRAM_RHO || MODE == GRAM_DELTA;
+    constexpr bool DIAG = MODE == GRAM_DIAG;
+    constexpr int kEpiThreads = NS * 128;
+    constexpr int kSliceCols = BN / NS;
+    constexpr int kChunks = kSliceCols / 32;           // 32-column chunks per warp
+    const GramArgs& g = k.g;
+    float *colw = sm.colw, *cola = sm.cola, *colrho = sm.colrho, *colx = sm.colx, *coly = sm.coly;
+    float *colred = sm.colred, *rowred = sm.rowred;
+    int *colidx = sm.colidx, *rowidx = sm.rowidx;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int e = threadIdx.x - 64;                    // 0 .. kEpiThreads - 1
+    const int quarter = warp & 3;                      // TMEM lane quarter this warp may read
+    const int slice = (warp - 2) >> 2;                 // which slice of the tile's columns this warp handles
+    const int rl = quarter * 32 + lane;                // tile-local row == TMEM lane
+    const int rows_out = g.row_end - g.row0;
+    const int b = call.b, ti = call.ti, tj = call.tj;
+    const int I0 = g.row0 + ti * BM, J0 = tj * BN;
+    const int i = I0 + rl;
+    const bool row_valid = SYM ? (i < g.n) : (i < g.row_end);
+    const size_t bo = (size_t)b * g.n;
+
+    // ---- per-column and per-row constants
+    for (int ce = e; ce < BN && !DIAG; ce += kEpiThreads) {
+        const int j = J0 + ce;
+        const bool cv = j < g.n;
+        colw[ce] = cv ? g.w[bo + j] : 0.f;
+        if (METRIC == 1) cola[ce] = cv ? g.a[bo + j] : 0.f;
+        if (MODE == GRAM_DELTA) {
+            colrho[ce] = cv ? g.rho[bo + j] : 0.f;
+            if (SPATIAL) {
+                colx[ce] = cv ? g.pos[2 * (bo + j)] : 0.f;
+                coly[ce] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
+            }
+        }
+    }
+    const float w_i = (row_valid && !DIAG) ? g.w[bo + i] : 0.f;
+    const float a_i = METRIC == 1 ? (row_valid ? g.a[bo + i] : 0.f) : 1.f;
+    const float m2w_i = -2.f * w_i;
+    float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
+    if (MODE == GRAM_DELTA && row_valid) {
+        rho_i = g.rho[bo + i];
+        if (SPATIAL) { x_i = g.pos[2 * (bo + i)]; y_i = g.pos[2 * (bo + i) + 1]; }
+    }
+    // every pair of the tile has i < j < n: no masking needed
+    const bool full = SYM && (J0 >= I0 + BM) && (J0 + BN <= g.n);
+
+    epi_bar_sync<kEpiThreads>();
+    if (ok && call.wait_bar) ok = mbar_wait(call.wait_bar, call.wait_parity, call.abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+
+    float racc = 0.f;                              // GRAM_RHO: row-side sum
+    float rbest = kInf;                            // GRAM_DELTA: row-side minimum and its tile-local column
+    int rbest_c = -1;
+    if (ok) {
+        tc_fence_after();
+        const uint32_t taddr = call.tmem_tile + ((uint32_t)(quarter * 32) << 16) + slice * kSliceCols;
+#pragma unroll 1
+        for (int c = 0; c < kChunks; ++c) {
+            float v[32];
+            tmem_ld32(taddr + c * 32, v);
+            if (c == kChunks - 1) {
+                // this thread has read all it needs from the accumulator
+                tc_fence_before();
+                if (call.arrive_bar) mbar_arrive(call.arrive_bar);
+            }
+            const int cl0 = slice * kSliceCols + c * 32;       // tile-local first column of the chunk
+            const float4* cw4 = reinterpret_cast<const float4*>(colw + cl0);
+            const float4* ca4 = reinterpret_cast<const float4*>(cola + cl0);
+            if (MODE == GRAM_DIAG) {
+                // g_ii sits in column rl of row rl: the chunk that starts at this warp's first row
+                if (cl0 == quarter * 32 && row_valid) {
+                    float gii = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) gii = (u == lane) ? v[u] : gii;
+                    // The squared norm comes from the same tensor-core arithmetic as every g_ij, so the
+                    // rounding of the accumulation cancels in s_ij = g_ij / sqrt(g_ii g_jj) where it
+                    // matters: near-duplicates (s -> 1, d^2 = 2 - 2 s -> 0); exact duplicates give s = 1.
+                    g.w_out[bo + i] = METRIC == 0 ? (gii > 0.f ? 1.0f / sqrtf(gii) : 0.f) : 1.f;
+                    g.a_out[bo + i] = METRIC == 0 ? 1.f : gii;
+                    if (g.best) g.best[bo + i] = ~0ull;
+                }
+            } else if (MODE == GRAM_SIM) {
+                if (row_valid) {
+                    float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) {
+                        const int j = J0 + cl0 + u;
+                        if (j < g.n) o[j] = METRIC == 0 ? (v[u] * w_i) * colw[cl0 + u] : v[u];
+                    }
+                }
+            } else if (MODE == GRAM_RHO) {
+                // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
+#pragma unroll
+                for (int q4 = 0; q4 < 8; ++q4) {
+                    const float4 cw = cw4[q4];
+                    float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (METRIC == 1) ca = ca4[q4];
+                    const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                    const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const int u = 4 * q4 + r;
+                        const float x = v[u] * cwv[r];
+                        const float base = METRIC == 0 ? 2.f : a_i + cav[r];
+                        const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                        v[u] = ex2_approx(d2 * g.c2);
+                    }
+                }
+                if (!full) {
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) {
+                        const int j = J0 + cl0 + u;
+                        v[u] = (j > i && j < g.n && row_valid) ? v[u] : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 32; ++u) racc += v[u];
+                const float cs = warp_transpose_reduce<false>(v, lane);
+                colred[quarter * BN + cl0 + lane] = cs;
+            } else {  // GRAM_DELTA, Eq. 3
+                const float4* cr4 = reinterpret_cast<const float4*>(colrho + cl0);
+                const float4* cx4 = reinterpret_cast<const float4*>(colx + cl0);
+                const float4* cy4 = reinterpret_cast<const float4*>(coly + cl0);
+                uint32_t kc[32];                   // column-side keys: d^2 >= 0 orders like its bit pattern
+#pragma unroll
+                for (int q4 = 0; q4 < 8; ++q4) {
+                    const float4 cw = cw4[q4];
+                    const float4 cr = cr4[q4];
+                    float4 ca = make_float4(0.f, 0.f, 0.f, 0.f), cx = ca, cy = ca;
+                    if (METRIC == 1) ca = ca4[q4];
+                    if (SPATIAL) { cx = cx4[q4]; cy = cy4[q4]; }
+                    const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                    const float crv[4] = {cr.x, cr.y, cr.z, cr.w};
+                    const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+                    const float cxv[4] = {cx.x, cx.y, cx.z, cx.w};
+                    const float cyv[4] = {cy.x, cy.y, cy.z, cy.w};
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const int u = 4 * q4 + r;
+                        const float x = v[u] * cwv[r];
+                        const float base = METRIC == 0 ? 2.f : a_i + cav[r];
+                        float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                        bool usable = true;        // the pair may serve as (child, parent) at all
+                        if (SPATIAL) {
+                            const float dx = cxv[r] - x_i, dy = cyv[r] - y_i;
+                            usable = fmaf(dx, dx, dy * dy) <= g.tau2;
+                        }
+                        if (!full) {
+                            const int j = J0 + cl0 + u;
+                            usable = usable && j > i && j < g.n && row_valid;
+                        }
+                        if (SPATIAL || !full) d2 = usable ? d2 : kInf;
+                        // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
+                        const bool jd = crv[r] > rho_i;
+                        const float kr = jd ? d2 : kInf;       // j as parent candidate of i (row side)
+                        kc[u] = __float_as_uint(jd ? kInf : d2);   // i as parent candidate of j (column side)
+                        if (kr < rbest) { rbest = kr; rbest_c = cl0 + u; }
+                    }
+                }
+                // column side: minimum over this warp's 32 rows and the lowest row that attains it
+                uint32_t my_min = 0x7f800000u, my_rows = 0;
+#pragma unroll
+                for (int u = 0; u < 32; ++u) {
+                    const uint32_t m = __reduce_min_sync(0xffffffffu, kc[u]);
+                    const uint32_t rows = __ballot_sync(0xffffffffu, kc[u] == m);
+                    if (lane == u) { my_min = m; my_rows = rows; }
+                }
+                colred[quarter * BN + cl0 + lane] = __uint_as_float(my_min);
+                colidx[quarter * BN + cl0 + lane] =
+                    my_min < 0x7f800000u ? I0 + quarter * 32 + (__ffs(my_rows) - 1) : -1;
+            }
+        }
+    }
+
+    if (SYM) {
+        // ---- combine the four column slices of every row and the four row quarters of every column
+        if (slice > 0) {
+            rowred[(slice - 1) * BM + rl] = MODE == GRAM_RHO ? racc : rbest;
+            if (MODE == GRAM_DELTA) rowidx[(slice - 1) * BM + rl] = rbest_c;
+        }
+        epi_bar_sync<kEpiThreads>();
+        if (ok) {
+            const int slot_base = b * k.t.slots();
+            if (MODE == GRAM_RHO) {
+                if (slice == 0 && row_valid) {
+#pragma unroll
+                    for (int q = 0; q < NS - 1; ++q) racc += rowred[q * BM + rl];       // fixed order
+                    g.part[((size_t)(slot_base + tj)) * k.t.n_pad + i] = racc;
+                }
+                for (int ce = e; ce < BN; ce += kEpiThreads)
+                    if (J0 + ce < g.n)
+                        g.part[((size_t)(slot_base + k.t.TJ + ti)) * k.t.n_pad + J0 + ce] =
+                            ((colred[ce] + colred[BN + ce]) + colred[2 * BN + ce]) + colred[3 * BN + ce];
+            } else {
+                if (slice == 0 && row_valid) {
+#pragma unroll
+                    for (int q = 0; q < NS - 1; ++q) {                             // ascending columns: ties keep the lower one
+                        const float other = rowred[q * BM + rl];
+                        if (other < rbest) { rbest = other; rbest_c = rowidx[q * BM + rl]; }
+                    }
+                    if (rbest_c >= 0) {
+                        const unsigned long long packed =
+                            ((unsigned long long)__float_as_uint(rbest) << 32) |
+                            (unsigned long long)(uint32_t)(J0 + rbest_c);
+                        atomicMin(g.best + bo + i, packed);
+                    }
+                }
+                for (int ce = e; ce < BN; ce += kEpiThreads) {
+                    if (J0 + ce >= g.n) continue;
+                    float bk = kInf;
+                    int bi = -1;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {                                  // ascending rows: ties keep the lower row
+                        const float kk = colred[q * BN + ce];
+                        if (kk < bk) { bk = kk; bi = colidx[q * BN + ce]; }
+                    }
+                    if (bi >= 0) {
+                        const unsigned long long packed =
+                            ((unsigned long long)__float_as_uint(bk) << 32) | (unsigned long long)(uint32_t)bi;
+                        atomicMin(g.best + bo + J0 + ce, packed);
+                    }
+                }
+            }
+        }
+    }
+    // shared arrays are rewritten for the next tile; all epilogue warps leave together or not at all
+    return epi_bar_or<kEpiThreads>(!ok);
+}
+
+// ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
 template <int BN, int MODE, int METRIC, bool SPATIAL>
@@ -377,233 +624,24 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2 ..)
-        const int e = threadIdx.x - 64;                    // 0 .. kEpiThreads - 1
-        const int quarter = warp & 3;                      // TMEM lane quarter this warp may read
-        const int slice = (warp - 2) >> 2;                 // which slice of the tile's columns this warp handles
-        const int rl = quarter * 32 + lane;                // tile-local row == TMEM lane
-        constexpr int kSliceCols = BN / NS;
-        constexpr int kChunks = kSliceCols / 32;           // 32-column chunks per warp
-        const int rows_out = g.row_end - g.row0;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
+        EpiSmem sm;
+        sm.colw = colw; sm.cola = cola; sm.colrho = colrho; sm.colx = colx; sm.coly = coly;
+        sm.colred = colred; sm.colidx = colidx; sm.rowred = rowred; sm.rowidx = rowidx;
 
         grid_dependency_wait();                            // w, a, rho, best come from the preceding kernels
 
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-            int b, ti, tj;
-            decode_tile<BN, SYM, DIAG>(k, t, b, ti, tj);
-            const int I0 = g.row0 + ti * BM, J0 = tj * BN;
-            const int i = I0 + rl;
-            const bool row_valid = SYM ? (i < g.n) : (i < g.row_end);
-            const size_t bo = (size_t)b * g.n;
-
-            // ---- per-column and per-row constants
-            for (int ce = e; ce < BN && !DIAG; ce += kEpiThreads) {
-                const int j = J0 + ce;
-                const bool cv = j < g.n;
-                colw[ce] = cv ? g.w[bo + j] : 0.f;
-                if (METRIC == 1) cola[ce] = cv ? g.a[bo + j] : 0.f;
-                if (MODE == GRAM_DELTA) {
-                    colrho[ce] = cv ? g.rho[bo + j] : 0.f;
-                    if (SPATIAL) {
-                        colx[ce] = cv ? g.pos[2 * (bo + j)] : 0.f;
-                        coly[ce] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
-                    }
-                }
-            }
-            const float w_i = (row_valid && !DIAG) ? g.w[bo + i] : 0.f;
-            const float a_i = METRIC == 1 ? (row_valid ? g.a[bo + i] : 0.f) : 1.f;
-            const float m2w_i = -2.f * w_i;
-            float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
-            if (MODE == GRAM_DELTA && row_valid) {
-                rho_i = g.rho[bo + i];
-                if (SPATIAL) { x_i = g.pos[2 * (bo + i)]; y_i = g.pos[2 * (bo + i) + 1]; }
-            }
-            // every pair of the tile has i < j < n: no masking needed
-            const bool full = SYM && (J0 >= I0 + BM) && (J0 + BN <= g.n);
-
-            epi_bar_sync<kEpiThreads>();
-            if (ok) ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-
-            float racc = 0.f;                              // GRAM_RHO: row-side sum
-            float rbest = kInf;                            // GRAM_DELTA: row-side minimum and its tile-local column
-            int rbest_c = -1;
-            if (ok) {
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + slice * kSliceCols;
-#pragma unroll 1
-                for (int c = 0; c < kChunks; ++c) {
-                    float v[32];
-                    tmem_ld32(taddr + c * 32, v);
-                    if (c == kChunks - 1) {
-                        // this thread has read all it needs from the accumulator
-                        tc_fence_before();
-                        mbar_arrive(bar_tempty + 8 * acc);
-                    }
-                    const int cl0 = slice * kSliceCols + c * 32;       // tile-local first column of the chunk
-                    const float4* cw4 = reinterpret_cast<const float4*>(colw + cl0);
-                    const float4* ca4 = reinterpret_cast<const float4*>(cola + cl0);
-                    if (MODE == GRAM_DIAG) {
-                        // g_ii sits in column rl of row rl: the chunk that starts at this warp's first row
-                        if (cl0 == quarter * 32 && row_valid) {
-                            float gii = 0.f;
-#pragma unroll
-                            for (int u = 0; u < 32; ++u) gii = (u == lane) ? v[u] : gii;
-                            // The squared norm comes from the same tensor-core arithmetic as every g_ij, so the
-                            // rounding of the accumulation cancels in s_ij = g_ij / sqrt(g_ii g_jj) where it
-                            // matters: near-duplicates (s -> 1, d^2 = 2 - 2 s -> 0); exact duplicates give s = 1.
-                            g.w_out[bo + i] = METRIC == 0 ? (gii > 0.f ? 1.0f / sqrtf(gii) : 0.f) : 1.f;
-                            g.a_out[bo + i] = METRIC == 0 ? 1.f : gii;
-                            if (g.best) g.best[bo + i] = ~0ull;
-                        }
-                    } else if (MODE == GRAM_SIM) {
-                        if (row_valid) {
-                            float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
-#pragma unroll
-                            for (int u = 0; u < 32; ++u) {
-                                const int j = J0 + cl0 + u;
-                                if (j < g.n) o[j] = METRIC == 0 ? (v[u] * w_i) * colw[cl0 + u] : v[u];
-                            }
-                        }
-                    } else if (MODE == GRAM_RHO) {
-                        // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
-#pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {
-                            const float4 cw = cw4[q4];
-                            float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (METRIC == 1) ca = ca4[q4];
-                            const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
-                            const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const int u = 4 * q4 + r;
-                                const float x = v[u] * cwv[r];
-                                const float base = METRIC == 0 ? 2.f : a_i + cav[r];
-                                const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
-                                v[u] = ex2_approx(d2 * g.c2);
-                            }
-                        }
-                        if (!full) {
-#pragma unroll
-                            for (int u = 0; u < 32; ++u) {
-                                const int j = J0 + cl0 + u;
-                                v[u] = (j > i && j < g.n && row_valid) ? v[u] : 0.f;
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < 32; ++u) racc += v[u];
-                        const float cs = warp_transpose_reduce<false>(v, lane);
-                        colred[quarter * BN + cl0 + lane] = cs;
-                    } else {  // GRAM_DELTA, Eq. 3
-                        const float4* cr4 = reinterpret_cast<const float4*>(colrho + cl0);
-                        const float4* cx4 = reinterpret_cast<const float4*>(colx + cl0);
-                        const float4* cy4 = reinterpret_cast<const float4*>(coly + cl0);
-                        uint32_t kc[32];                   // column-side keys: d^2 >= 0 orders like its bit pattern
-#pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {
-                            const float4 cw = cw4[q4];
-                            const float4 cr = cr4[q4];
-                            float4 ca = make_float4(0.f, 0.f, 0.f, 0.f), cx = ca, cy = ca;
-                            if (METRIC == 1) ca = ca4[q4];
-                            if (SPATIAL) { cx = cx4[q4]; cy = cy4[q4]; }
-                            const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
-                            const float crv[4] = {cr.x, cr.y, cr.z, cr.w};
-                            const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
-                            const float cxv[4] = {cx.x, cx.y, cx.z, cx.w};
-                            const float cyv[4] = {cy.x, cy.y, cy.z, cy.w};
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                const int u = 4 * q4 + r;
-                                const float x = v[u] * cwv[r];
-                                const float base = METRIC == 0 ? 2.f : a_i + cav[r];
-                                float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
-                                bool usable = true;        // the pair may serve as (child, parent) at all
-                                if (SPATIAL) {
-                                    const float dx = cxv[r] - x_i, dy = cyv[r] - y_i;
-                                    usable = fmaf(dx, dx, dy * dy) <= g.tau2;
-                                }
-                                if (!full) {
-                                    const int j = J0 + cl0 + u;
-                                    usable = usable && j > i && j < g.n && row_valid;
-                                }
-                                if (SPATIAL || !full) d2 = usable ? d2 : kInf;
-                                // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
-                                const bool jd = crv[r] > rho_i;
-                                const float kr = jd ? d2 : kInf;       // j as parent candidate of i (row side)
-                                kc[u] = __float_as_uint(jd ? kInf : d2);   // i as parent candidate of j (column side)
-                                if (kr < rbest) { rbest = kr; rbest_c = cl0 + u; }
-                            }
-                        }
-                        // column side: minimum over this warp's 32 rows and the lowest row that attains it
-                        uint32_t my_min = 0x7f800000u, my_rows = 0;
-#pragma unroll
-                        for (int u = 0; u < 32; ++u) {
-                            const uint32_t m = __reduce_min_sync(0xffffffffu, kc[u]);
-                            const uint32_t rows = __ballot_sync(0xffffffffu, kc[u] == m);
-                            if (lane == u) { my_min = m; my_rows = rows; }
-                        }
-                        colred[quarter * BN + cl0 + lane] = __uint_as_float(my_min);
-                        colidx[quarter * BN + cl0 + lane] =
-                            my_min < 0x7f800000u ? I0 + quarter * 32 + (__ffs(my_rows) - 1) : -1;
-                    }
-                }
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-            }
-
-            if (SYM) {
-                // ---- combine the four column slices of every row and the four row quarters of every column
-                if (slice > 0) {
-                    rowred[(slice - 1) * BM + rl] = MODE == GRAM_RHO ? racc : rbest;
-                    if (MODE == GRAM_DELTA) rowidx[(slice - 1) * BM + rl] = rbest_c;
-                }
-                epi_bar_sync<kEpiThreads>();
-                if (ok) {
-                    const int slot_base = b * k.t.slots();
-                    if (MODE == GRAM_RHO) {
-                        if (slice == 0 && row_valid) {
-#pragma unroll
-                            for (int q = 0; q < NS - 1; ++q) racc += rowred[q * BM + rl];       // fixed order
-                            g.part[((size_t)(slot_base + tj)) * k.t.n_pad + i] = racc;
-                        }
-                        for (int ce = e; ce < BN; ce += kEpiThreads)
-                            if (J0 + ce < g.n)
-                                g.part[((size_t)(slot_base + k.t.TJ + ti)) * k.t.n_pad + J0 + ce] =
-                                    ((colred[ce] + colred[BN + ce]) + colred[2 * BN + ce]) + colred[3 * BN + ce];
-                    } else {
-                        if (slice == 0 && row_valid) {
-#pragma unroll
-                            for (int q = 0; q < NS - 1; ++q) {                             // ascending columns: ties keep the lower one
-                                const float other = rowred[q * BM + rl];
-                                if (other < rbest) { rbest = other; rbest_c = rowidx[q * BM + rl]; }
-                            }
-                            if (rbest_c >= 0) {
-                                const unsigned long long packed =
-                                    ((unsigned long long)__float_as_uint(rbest) << 32) |
-                                    (unsigned long long)(uint32_t)(J0 + rbest_c);
-                                atomicMin(g.best + bo + i, packed);
-                            }
-                        }
-                        for (int ce = e; ce < BN; ce += kEpiThreads) {
-                            if (J0 + ce >= g.n) continue;
-                            float bk = kInf;
-                            int bi = -1;
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {                                  // ascending rows: ties keep the lower row
-                                const float kk = colred[q * BN + ce];
-                                if (kk < bk) { bk = kk; bi = colidx[q * BN + ce]; }
-                            }
-                            if (bi >= 0) {
-                                const unsigned long long packed =
-                                    ((unsigned long long)__float_as_uint(bk) << 32) | (unsigned long long)(uint32_t)bi;
-                                atomicMin(g.best + bo + J0 + ce, packed);
-                            }
-                        }
-                    }
-                }
-            }
-            // shared arrays are rewritten for the next tile; all epilogue warps leave together or not at all
-            if (epi_bar_or<kEpiThreads>(!ok)) break;
+            EpiCall c;
+            decode_tile<BN, SYM, DIAG>(k, t, c.b, c.ti, c.tj);
+            c.tmem_tile = tmem_base + acc * BN;
+            c.wait_bar = bar_tfull + 8 * acc;
+            c.wait_parity = acc_phase;
+            c.arrive_bar = bar_tempty + 8 * acc;
+            c.abort_flag = abort_flag;
+            if (epi_tile<BN, MODE, METRIC, SPATIAL, NS>(k, sm, c, ok)) break;
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
 
