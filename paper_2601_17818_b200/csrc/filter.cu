@@ -31,12 +31,7 @@ __global__ void rho_reduce_kernel(const float* __restrict__ part, int n, GramTil
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int b = blockIdx.y;
     if (i >= n) return;
-    const float* p = part + (size_t)b * t.slots() * t.n_pad + i;
-    const int ti = i / BM, tj = i / t.BN;
-    float s = 0.f;
-    for (int c = ti / t.R; c < t.TJ; ++c) s += p[(size_t)c * t.n_pad];
-    const int rows = min(t.TI, t.R * (tj + 1));
-    for (int r = 0; r < rows; ++r) s += p[(size_t)(t.TJ + r) * t.n_pad];
+    const float s = rho_from_partials(part + (size_t)b * t.slots() * t.n_pad + i, t, i);
     rho[(size_t)b * n + i] = s;
     if (rho_user) rho_user[(size_t)b * n + i] = s;
 }
@@ -312,22 +307,32 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     g.w_out = w; g.a_out = a;
     g.sim_out = nullptr; g.status = reinterpret_cast<int*>(ws);
 
-    // first kernel of the call: launched without programmatic overlap, so everything queued before the call
-    // (the producer of the features included) has completed when it starts
-    int rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
-    if (rc != VITCOP_OK) return rc;
-    rc = launch_gram_sweep(GRAM_RHO, feat, g, tiling, stream, true);
-    if (rc != VITCOP_OK) return rc;
-    {
-        cudaLaunchConfig_t cfg;
-        cudaLaunchAttribute attr[1];
-        pdl_config(cfg, attr, dim3((n + 255) / 256, B), dim3(256), 0, stream, true);
-        KernelTimeScope timed("rho_reduce_kernel", stream);
-        rc = record_cuda(cudaLaunchKernelEx(&cfg, rho_reduce_kernel, (const float*)part, n, tiling, rho, rho_user));
+    // The first kernel of the call is launched without programmatic overlap, so everything queued before the call
+    // (the producer of the features included) has completed when it starts.
+    int rc;
+    const bool resident = gram_fits_resident(B, n);
+    if (resident) {
+        g.rho_out = rho;
+        g.rho_user = rho_user;
+        g.grid_sync = reinterpret_cast<unsigned int*>(ws) + 2;       // zeroed with the status word at the start of the call
+        rc = launch_gram_resident(feat, g, make_gram_tiling(n, 128), stream);
+        if (rc != VITCOP_OK) return rc;
+    } else {
+        rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
+        if (rc != VITCOP_OK) return rc;
+        rc = launch_gram_sweep(GRAM_RHO, feat, g, tiling, stream, true);
+        if (rc != VITCOP_OK) return rc;
+        {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[1];
+            pdl_config(cfg, attr, dim3((n + 255) / 256, B), dim3(256), 0, stream, true);
+            KernelTimeScope timed("rho_reduce_kernel", stream);
+            rc = record_cuda(cudaLaunchKernelEx(&cfg, rho_reduce_kernel, (const float*)part, n, tiling, rho, rho_user));
+            if (rc != VITCOP_OK) return rc;
+        }
+        rc = launch_gram_sweep(GRAM_DELTA, feat, g, tiling, stream, true);
         if (rc != VITCOP_OK) return rc;
     }
-    rc = launch_gram_sweep(GRAM_DELTA, feat, g, tiling, stream, true);
-    if (rc != VITCOP_OK) return rc;
 
     const int nc = n_centers < n ? n_centers : n;
     const size_t smem = (size_t)n * 8 + (((size_t)n + 15) & ~(size_t)15) + (size_t)(nc > 0 ? nc : 1) * 4 + 16;

@@ -256,6 +256,7 @@ struct EpiCall {
     uint32_t tmem_tile;            // TMEM address (lane 0) of the tile's first accumulator column
     uint32_t wait_bar, wait_parity;   // mbarrier that completes when the accumulator is ready (0: it already is)
     uint32_t arrive_bar;           // mbarrier to arrive on once this thread has read the accumulator (0: none)
+    bool rho_from_part;            // GRAM_DELTA: sum rho from the density partials (and publish it from diagonal tiles)
     volatile int* abort_flag;
 };
 
@@ -290,7 +291,19 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
         colw[ce] = cv ? g.w[bo + j] : 0.f;
         if (METRIC == 1) cola[ce] = cv ? g.a[bo + j] : 0.f;
         if (MODE == GRAM_DELTA) {
-            colrho[ce] = cv ? g.rho[bo + j] : 0.f;
+            float rj = 0.f;
+            if (cv) {
+                if (call.rho_from_part) {
+                    rj = rho_from_partials(g.part + (size_t)b * k.t.slots() * k.t.n_pad + j, k.t, j);
+                    if (ti == tj) {                        // the diagonal tile of a row block publishes its tokens' rho
+                        g.rho_out[bo + j] = rj;
+                        if (g.rho_user) g.rho_user[bo + j] = rj;
+                    }
+                } else {
+                    rj = g.rho[bo + j];
+                }
+            }
+            colrho[ce] = rj;
             if (SPATIAL) {
                 colx[ce] = cv ? g.pos[2 * (bo + j)] : 0.f;
                 coly[ce] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
@@ -302,7 +315,8 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
     const float m2w_i = -2.f * w_i;
     float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
     if (MODE == GRAM_DELTA && row_valid) {
-        rho_i = g.rho[bo + i];
+        rho_i = call.rho_from_part ? rho_from_partials(g.part + (size_t)b * k.t.slots() * k.t.n_pad + i, k.t, i)
+                                   : g.rho[bo + i];
         if (SPATIAL) { x_i = g.pos[2 * (bo + i)]; y_i = g.pos[2 * (bo + i) + 1]; }
     }
     // every pair of the tile has i < j < n: no masking needed
@@ -639,6 +653,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             c.wait_bar = bar_tfull + 8 * acc;
             c.wait_parity = acc_phase;
             c.arrive_bar = bar_tempty + 8 * acc;
+            c.rho_from_part = false;
             c.abort_flag = abort_flag;
             if (epi_tile<BN, MODE, METRIC, SPATIAL, NS>(k, sm, c, ok)) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -652,6 +667,216 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tmem_dealloc(tmem_base, kTmemCols);
     }
     if (threadIdx.x == 0 && *abort_flag && g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// the resident kernel: density and delta from ONE pass over the Gram tiles (small problems)
+// ------------------------------------------------------------------------------------------------
+// Every CTA owns at most kResidentSlots tiles of 128 x 128 and keeps all their accumulators in tensor memory
+// (4 x 128 of the 512 columns).  Phases of the epilogue warps:
+//   0. the diagonal tiles yield g_ii -> per-token normalisation factors; grid-wide barrier
+//   1. density epilogue of every tile -> rho partials; grid-wide barrier
+//   2. delta epilogue of every tile, re-reading the accumulators; rho of the tile's rows and columns is summed
+//      from the partials on the way (the diagonal tiles publish it)
+// The grid (at most one CTA per SM) is launched cooperatively, so all CTAs are resident together; the barriers
+// are counters in global memory with a bounded wait.  Dependents are released only at the very end: released
+// earlier, their CTAs could take the SM slots that CTAs of this grid still wait for.
+constexpr int kResidentSlots = 4;
+constexpr int kResidentEpiThreads = 512;
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Barrier over all CTAs of the grid, called by the epilogue threads.  Returns true when the grid must give up.
+__device__ __forceinline__ bool resident_grid_barrier(unsigned int* counter, volatile int* abort_flag, bool aborted) {
+    __threadfence();                                       // this thread's global writes are visible device-wide
+    epi_bar_sync<kResidentEpiThreads>();
+    if (threadIdx.x == 64 && !aborted) {
+        atomicAdd(counter, 1u);
+        const unsigned long long t0 = global_ns();
+        while (ld_acquire_u32(counter) < gridDim.x) {
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+        }
+    }
+    const bool stop = epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
+    __threadfence();
+    return stop;
+}
+
+template <int METRIC, bool SPATIAL>
+__global__ void __launch_bounds__(64 + kResidentEpiThreads, 1)
+gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const KernelArgs k) {
+    constexpr int BN = BM;
+    constexpr int NS = 4;
+    using S = GemmSmem<BN>;
+    const GramArgs& g = k.g;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (tiles - raw);
+    EpiSmem sm;
+    sm.colw = reinterpret_cast<float*>(gen + S::kTileBytes);
+    sm.cola = sm.colw + BN;
+    sm.colrho = sm.cola + BN;
+    sm.colx = sm.colrho + BN;
+    sm.coly = sm.colx + BN;
+    sm.colred = sm.coly + BN;
+    sm.colidx = reinterpret_cast<int*>(sm.colred + 4 * BN);
+    sm.rowred = reinterpret_cast<float*>(sm.colidx + 4 * BN);
+    sm.rowidx = reinterpret_cast<int*>(sm.rowred + 3 * BM);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
+    // barriers: full[kStages], empty[kStages], tmem_full[kResidentSlots], drain
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * S::kStages;
+    const uint32_t bar_tfull = bar_empty + 8 * S::kStages;
+    const uint32_t bar_drain = bar_tfull + 8 * kResidentSlots;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + kResidentSlots + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr uint32_t kTmemCols = kResidentSlots * BN;   // 512: the whole tensor memory of the SM
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S::kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < kResidentSlots; ++a) mbar_init(bar_tfull + 8 * a, 1);
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const long long total_tiles = k.total_tiles;          // <= kResidentSlots * gridDim.x (checked by the launcher)
+    const int KB = g.D / BK;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0, issued_parity = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+                int b, ti, tj;
+                decode_tile<BN, true, false>(k, t, b, ti, tj);
+                const int I0 = ti * BM, J0 = tj * BN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = tiles + stage * S::kStageBytes;
+                    mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
+                    tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
+                    tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
+                    issued |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                for (int s = 0; s < S::kStages; ++s)
+                    if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer: tile s of this CTA -> slot s
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            uint32_t stage = 0, phase = 0;
+            uint32_t slot = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x, ++slot) {
+                const uint32_t d_tmem = tmem_base + slot * BN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = tiles + stage * S::kStageBytes;
+                    const uint64_t da = umma_desc_k128(sa), db = umma_desc_k128(sa + S::kABytes);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk), idesc,
+                                    (kb > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(bar_empty + 8 * stage);
+                    if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(bar_tfull + 8 * slot);
+            }
+            if (!ok) {
+                tc_commit(bar_drain);
+                mbar_drain(bar_drain, 0);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..17)
+        const int e = threadIdx.x - 64;
+        bool ok = true;
+        bool stop = false;
+        grid_dependency_wait();
+
+        // ---- phase 0: the diagonal tiles give g_ii, hence the per-token factors every other epilogue needs
+        uint32_t slot = 0;
+        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
+            EpiCall c;
+            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            if (c.ti != c.tj) continue;                    // uniform over the CTA
+            c.tmem_tile = tmem_base + slot * BN;
+            c.wait_bar = bar_tfull + 8 * slot;
+            c.wait_parity = 0;
+            c.arrive_bar = 0;
+            c.rho_from_part = false;
+            c.abort_flag = abort_flag;
+            stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS>(k, sm, c, ok);
+        }
+        stop = resident_grid_barrier(g.grid_sync + 1, abort_flag, stop);
+        // ---- phase 1: density partials
+        slot = 0;
+        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
+            EpiCall c;
+            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            c.tmem_tile = tmem_base + slot * BN;
+            c.wait_bar = bar_tfull + 8 * slot;
+            c.wait_parity = 0;
+            c.arrive_bar = 0;
+            c.rho_from_part = false;
+            c.abort_flag = abort_flag;
+            stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS>(k, sm, c, ok);
+        }
+        stop = resident_grid_barrier(g.grid_sync, abort_flag, stop);
+        // ---- phase 2: delta and parents from the same accumulators; every tile sums the rho of its own rows and
+        //      columns from the partials (fixed order: the same bits everywhere)
+        slot = 0;
+        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
+            EpiCall c;
+            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            c.tmem_tile = tmem_base + slot * BN;
+            c.wait_bar = 0;
+            c.wait_parity = 0;
+            c.arrive_bar = 0;
+            c.rho_from_part = true;
+            c.abort_flag = abort_flag;
+            stop = epi_tile<BN, GRAM_DELTA, METRIC, SPATIAL, NS>(k, sm, c, ok);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && *abort_flag && g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+    grid_dependency_launch_dependents();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -750,6 +975,33 @@ int launch_bn(int mode, const CUtensorMap& ma, const CUtensorMap& mb, const Kern
     }
 }
 
+
+template <int METRIC, bool SPATIAL>
+int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream) {
+    using S = GemmSmem<BM>;
+    static bool attr_done = false;
+    auto kern = gram_resident_kernel<METRIC, SPATIAL>;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal);
+        if (e != cudaSuccess) return record_cuda(e);
+        attr_done = true;
+    }
+    const long long ctas = (k.total_tiles + kResidentSlots - 1) / kResidentSlots;
+    cudaLaunchConfig_t cfg = {};
+    // as many CTAs as there are SMs (never fewer than the tiles need): the shortest chain of tiles per CTA
+    cfg.gridDim = dim3((unsigned)(k.total_tiles < num_sms() ? k.total_tiles : (ctas > num_sms() ? ctas : num_sms())));
+    cfg.blockDim = dim3(64 + kResidentEpiThreads);
+    cfg.dynamicSmemBytes = S::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;          // all CTAs resident together: they wait for one another
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    KernelTimeScope timed("gram_resident_kernel", stream);
+    return record_cuda(cudaLaunchKernelEx(&cfg, kern, ma, mb, k));
+}
+
 }  // namespace
 
 int gram_pick_bn(int B, int n) {
@@ -782,6 +1034,38 @@ int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const Gr
         return VITCOP_ERR_CUDA;
     return tiling.BN == 256 ? launch_bn<256>(mode, ma, mb, k, stream, pdl)
                             : launch_bn<128>(mode, ma, mb, k, stream, pdl);
+}
+
+bool gram_fits_resident(int B, int n) {
+    static int cooperative = -1;                          // the resident kernel needs a cooperative launch
+    if (cooperative < 0) {
+        int dev = 0, v = 0;
+        cooperative = (cudaGetDevice(&dev) == cudaSuccess &&
+                       cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 0;
+    }
+    if (!cooperative) return false;
+    const long long ti = (n + BM - 1) / BM;
+    const long long tiles = (long long)B * ti * (ti + 1) / 2;
+    return tiles > 0 && tiles <= (long long)kResidentSlots * num_sms();
+}
+
+int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream) {
+    KernelArgs k;
+    k.g = args;
+    k.t = tiling;
+    k.g.row0 = 0;
+    k.g.row_end = args.n;
+    k.total_tiles = (long long)args.B * k.t.tiles_per_b;
+    if (k.total_tiles <= 0) return VITCOP_OK;
+    if (tiling.BN != BM || k.total_tiles > (long long)kResidentSlots * num_sms()) return VITCOP_ERR_INVALID_ARG;
+    CUtensorMap ma, mb;
+    if (!make_feat_map(&ma, feat, args.B, args.n, args.D, BM) || !make_feat_map(&mb, feat, args.B, args.n, args.D, BM))
+        return VITCOP_ERR_CUDA;
+    const bool euclid = args.metric == 1;
+    const bool spatial = args.tau2 >= 0.f && args.pos != nullptr;
+    if (spatial)
+        return euclid ? launch_resident_one<1, true>(ma, mb, k, stream) : launch_resident_one<0, true>(ma, mb, k, stream);
+    return euclid ? launch_resident_one<1, false>(ma, mb, k, stream) : launch_resident_one<0, false>(ma, mb, k, stream);
 }
 
 }  // namespace vitcop

@@ -54,8 +54,43 @@ struct GramArgs {
     float* sim_out;             // [B, row_end - row0, n]          (GRAM_SIM)
     float* w_out;               // [B, n] factors written by GRAM_DIAG (best, if given, is reset to ~0 as well)
     float* a_out;               // [B, n]
+    float* rho_out;             // [B, n] written by the resident sweep (same memory as rho)
+    float* rho_user;            // [B, n] optional copy of rho for the caller
+    unsigned int* grid_sync;    // two zeroed counters for the resident sweep's grid-wide barriers
     int* status;                // device status word
 };
+
+// rho of token i of one sample from the partial sums of the tiles that hold it, in a fixed order (reproducible
+// bits): the row-side slots of the column tiles that pair row tile i / 128 with later tokens, then the column-side
+// slots of the row tiles that pair column tile i / BN with earlier tokens.  `p` points at the sample's slot 0, token i.
+__host__ __device__ inline float rho_from_partials(const float* p, const GramTiling& t, int i) {
+    const int ti = i / kGramBM, tj = i / t.BN;
+    const int cap = t.R * (tj + 1);
+    const int rows = t.TI < cap ? t.TI : cap;
+    // slots [c0, TJ) on the row side, then [TJ, TJ + rows) on the column side: one contiguous walk, loaded eight
+    // at a time (independent loads) and added one by one in slot order
+    const int first = ti / t.R, last = t.TJ + rows;
+    float s = 0.f;
+    for (int c = first; c < last; c += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = (c + u < last) ? p[(size_t)(c + u) * t.n_pad] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (c + u < last) s += v[u];
+    }
+    return s;
+}
+
+// True when the whole symmetric sweep of the problem fits the tensor memory of one wave of CTAs (at most four
+// 128 x 128 tiles per SM): density and delta can then share one pass over the Gram tiles (launch_gram_resident).
+bool gram_fits_resident(int B, int n);
+
+// One kernel for the norms, Eq. 2 and Eq. 3 on small problems: every CTA keeps the accumulators of its tiles in
+// tensor memory; the grid synchronises (bounded waits) after the diagonal tiles have produced the per-token
+// factors and after the density partials; the delta epilogue sums the partials it needs itself and re-reads the
+// same accumulators.  `tiling` = make_gram_tiling(n, 128).
+int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream);
 
 // Enqueues one sweep.  `tiling` must come from make_gram_tiling(n, gram_pick_bn(B, n)) for the symmetric modes.
 int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream,
