@@ -52,6 +52,7 @@ extern "C" {
 #define VITCOP_OP_SIMILARITY  5
 #define VITCOP_OP_SALIENCY    6   /* vitcop_cls_saliency: B = images, H = heads, N = keys per head (M) */
 #define VITCOP_OP_MERGE       7   /* vitcop_merge_clusters: Nv = Nv_cap, N = Mcap */
+#define VITCOP_OP_COLLAB_STEP 8   /* vitcop_collaborative_step */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* vitcop_status_string(int status);
@@ -216,6 +217,27 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V,
                       int32_t* kept_pos, int32_t* out_len,
                       float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- Stage II in one call
+ * Algorithm 1 at layer l_s: VIC(F, P) -> cluster labels, K-norms (Eq. 4), collaborative pruning under the budget
+ * (Eq. 5, Algorithm 3 up to the elite set) and compaction of hidden states, K and V -- the work of
+ * vitcop_redundancy_filter followed by vitcop_prune_step with those labels, with identical results.  Being one
+ * call, it may run the K-norm, which does not depend on the clustering, beside the clustering's sweep instead of
+ * after it.  Every sample has the same Nv visual tokens at [vis_start, vis_start + Nv).
+ *   feat bf16 [B, Nv, D], pos fp32 [B, Nv, 2] or NULL, fp (host) as in vitcop_redundancy_filter
+ *   hidden, K, V, the outputs, kept_pos, out_len as in vitcop_prune_step (Nv_cap = Nv)
+ *   label_out int32 [B, Nv] and n_clusters_out int32 [B]: required outputs (the labels the selection used)
+ *   score_out, keep_idx_out [B, Nv], n_keep_out [B]: optional
+ *   workspace: vitcop_workspace_bytes(VITCOP_OP_COLLAB_STEP, B, 0, 0, 0, Nv, D, 0) bytes; one status word
+ * Errors: as the two calls it replaces. */
+int vitcop_collaborative_step(const void* feat, const float* pos, int D, const vitcop_filter_params* fp,
+                              const void* hidden, const void* K, const void* V,
+                              int B, int H, int N, int d, int Dh, int vis_start, int Nv, int budget,
+                              void* hidden_out, void* K_out, void* V_out, int Ncap,
+                              int32_t* kept_pos, int32_t* out_len,
+                              int32_t* label_out, int32_t* n_clusters_out,
+                              float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out,
+                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------- cluster merge
  * Eq. 6 of the paper (second half of Algorithm 3): in every cluster the tokens that were NOT kept as elites are

@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvitcop.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT = range(7)
-OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY, OP_MERGE = range(8)
+OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY, OP_MERGE, OP_COLLAB_STEP = range(9)
 MAX_VISUAL_TOKENS = 16384
 
 EXPORTS = [
@@ -27,6 +27,7 @@ EXPORTS = [
     "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
     "vitcop_prune_step_static", "vitcop_merge_clusters", "vitcop_cls_saliency", "vitcop_stage_count",
     "vitcop_flops_layer", "vitcop_visual_tokens_at_layer", "vitcop_flops_total", "vitcop_cr_int",
+    "vitcop_collaborative_step",
 ]
 
 
@@ -92,6 +93,9 @@ def lib() -> C.CDLL:
         L.vitcop_flops_total.restype = f64
         L.vitcop_cr_int.argtypes = [f64, f64, f64, i32, i32, i32]
         L.vitcop_cr_int.restype = f64
+        L.vitcop_collaborative_step.argtypes = [vp, vp, i32, C.POINTER(FilterParams), vp, vp, vp, i32, i32, i32, i32,
+                                                i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz,
+                                                vp]
         L.vitcop_kernel_timing_begin.argtypes = []
         L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
@@ -222,6 +226,25 @@ def vitcop_prune_step_static(hidden, K, V, vis_start: int, vis_len, Nv_cap: int,
                                         _ptr(V_out), Ncap, _ptr(kept_pos), _ptr(out_len), _ptr(score_out),
                                         _ptr(keep_idx_out), _ptr(n_keep_out), _stream())
     _check(rc, "vitcop_prune_step_static")
+    return out_len
+
+
+def vitcop_collaborative_step(feat, pos, hidden, K, V, vis_start: int, budget: int, hidden_out, K_out, V_out, out_len,
+                              label_out, n_clusters_out, workspace, metric: int = 0, d_c: float = 0.5, tau: float = 0.6,
+                              alpha: float = 0.05, n_centers: int = 0, kept_pos=None, score_out=None, keep_idx_out=None,
+                              n_keep_out=None):
+    """Stage II in one call: redundancy filter + fused pruning step in quota mode, K-norm beside the clustering."""
+    B, Nv, D = feat.shape
+    _, H, N, d = K.shape
+    Ncap = K_out.shape[2] if K_out is not None else hidden_out.shape[1]
+    Dh = hidden.shape[2] if hidden is not None else 0
+    p = FilterParams(int(metric), float(d_c), float(tau), float(alpha), int(n_centers))
+    rc = lib().vitcop_collaborative_step(_ptr(feat), _ptr(pos), D, C.byref(p), _ptr(hidden), _ptr(K), _ptr(V), B, H, N,
+                                         d, Dh, vis_start, Nv, int(budget), _ptr(hidden_out), _ptr(K_out), _ptr(V_out),
+                                         Ncap, _ptr(kept_pos), _ptr(out_len), _ptr(label_out), _ptr(n_clusters_out),
+                                         _ptr(score_out), _ptr(keep_idx_out), _ptr(n_keep_out), _ptr(workspace),
+                                         workspace.numel(), _stream())
+    _check(rc, "vitcop_collaborative_step")
     return out_len
 
 

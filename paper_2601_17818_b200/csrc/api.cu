@@ -189,6 +189,9 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
         case VITCOP_OP_COMPACT: *bytes = 0; return VITCOP_OK;
         case VITCOP_OP_SELECT: *bytes = kStatusBytes; return VITCOP_OK;
         case VITCOP_OP_PRUNE_STEP: *bytes = StepWs(B, Nv).total; return VITCOP_OK;
+        case VITCOP_OP_COLLAB_STEP:
+            *bytes = align_up(filter_workspace_bytes(B, Nv, D), 256) + StepWs(B, Nv).total;
+            return VITCOP_OK;
         case VITCOP_OP_MERGE:
             if (N < 0) return VITCOP_ERR_INVALID_ARG;
             *bytes = merge_workspace_bytes(B, Nv, N);
@@ -313,6 +316,52 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, i
     if (rc != VITCOP_OK) return rc;
     return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep, Nv_cap,
                           nkeep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, s, true);
+}
+
+int vitcop_collaborative_step(const void* feat, const float* pos, int D, const vitcop_filter_params* fp,
+                              const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
+                              int vis_start, int Nv, int budget, void* hidden_out, void* K_out, void* V_out, int Ncap,
+                              int32_t* kept_pos, int32_t* out_len, int32_t* label_out, int32_t* n_clusters_out,
+                              float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    if (!feat || !fp || !K || !out_len || !label_out || !n_clusters_out || budget < 0 || Nv < 0 || D < 0)
+        return VITCOP_ERR_INVALID_ARG;
+    if (fp->metric != 0 && fp->metric != 1) return VITCOP_ERR_INVALID_ARG;
+    if (!(fp->d_c > 0.f)) return VITCOP_ERR_INVALID_ARG;
+    int rc = check_compact_args(hidden, K, V, B, H, N, d, Dh, vis_start, nullptr, Nv, hidden_out, K_out, V_out, Ncap);
+    if (rc != VITCOP_OK) return rc;
+    rc = check_span(N, vis_start, nullptr, Nv, Nv);
+    if (rc != VITCOP_OK) return rc;
+    if (D % 64 || !aligned16(feat) || Nv > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
+    const size_t filter_bytes = align_up(filter_workspace_bytes(B, Nv, D), 256);
+    const StepWs lay(B, Nv);
+    if (!workspace || workspace_bytes < filter_bytes + lay.total || !aligned256(workspace)) return VITCOP_ERR_WORKSPACE;
+    int nc = fp->n_centers;
+    if (nc <= 0) {
+        const double v = std::ceil((double)Nv * fp->alpha);
+        nc = v < 0 ? 0 : (v > Nv ? Nv : (int)v);
+    }
+    if (nc > Nv) nc = Nv;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    char* ws2 = ws + filter_bytes;
+    float* score = score_out ? score_out : reinterpret_cast<float*>(ws2 + lay.off_score);
+    int32_t* keep = keep_idx_out ? keep_idx_out : reinterpret_cast<int32_t*>(ws2 + lay.off_keep);
+    int32_t* nkeep = n_keep_out ? n_keep_out : reinterpret_cast<int32_t*>(ws2 + lay.off_nkeep);
+    rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    if (B == 0) return VITCOP_OK;
+    if (Nv > 0) {
+        const KnormJob job = {K, B, H, N, d, vis_start, Nv, score};
+        rc = launch_filter(feat, pos, B, Nv, D, *fp, nc, label_out, n_clusters_out, nullptr, nullptr, nullptr, workspace,
+                           s, &job);
+        if (rc != VITCOP_OK) return rc;
+    }
+    rc = launch_select(score, label_out, B, nullptr, Nv, Nv, 1, 0, budget, keep, Nv, nkeep, nullptr,
+                       reinterpret_cast<int*>(ws), s, true);
+    if (rc != VITCOP_OK) return rc;
+    return launch_compact(hidden, K, V, B, H, N, d, Dh, nullptr, vis_start, nullptr, Nv, keep, Nv, nkeep, hidden_out,
+                          K_out, V_out, Ncap, kept_pos, out_len, s, true);
 }
 
 int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh, int vis_start, const int32_t* vis_len,

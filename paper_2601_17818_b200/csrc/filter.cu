@@ -289,7 +289,7 @@ size_t similarity_workspace_bytes(int B, int n, int D) {
 
 int launch_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params& p,
                   int n_centers, int32_t* label, int32_t* n_clusters, float* rho_user, float* delta2_user,
-                  int32_t* parent_user, void* workspace, cudaStream_t stream) {
+                  int32_t* parent_user, void* workspace, cudaStream_t stream, const KnormJob* knorm) {
     FilterWs l(B, n);
     char* ws = static_cast<char*>(workspace);
     float* w = reinterpret_cast<float*>(ws + l.off_w);
@@ -331,6 +331,15 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
             if (rc != VITCOP_OK) return rc;
         }
         rc = launch_gram_sweep(GRAM_DELTA, feat, g, tiling, stream, true);
+        if (rc != VITCOP_OK) return rc;
+    }
+
+    if (knorm) {
+        // The sweep before this point has released its dependents early: the K-norm streams K from HBM while the
+        // sweep's tensor-core and epilogue work goes on, and waits for the sweep before it ends.
+        rc = launch_knorm(knorm->K, knorm->B, knorm->H, knorm->d, (int64_t)knorm->H * knorm->N * knorm->d,
+                          (int64_t)knorm->N * knorm->d, knorm->d, knorm->vis_start, nullptr, knorm->Nv, knorm->score,
+                          knorm->Nv, stream, true);
         if (rc != VITCOP_OK) return rc;
     }
 

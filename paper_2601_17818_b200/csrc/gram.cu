@@ -680,8 +680,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 //   2. delta epilogue of every tile, re-reading the accumulators; rho of the tile's rows and columns is summed
 //      from the partials on the way (the diagonal tiles publish it)
 // The grid (at most one CTA per SM) is launched cooperatively, so all CTAs are resident together; the barriers
-// are counters in global memory with a bounded wait.  Dependents are released only at the very end: released
-// earlier, their CTAs could take the SM slots that CTAs of this grid still wait for.
+// are counters in global memory with a bounded wait.  Dependents are released after the first barrier, when every
+// CTA is known to be resident: released earlier, their CTAs could take SM slots that CTAs of this grid still need.
 constexpr int kResidentSlots = 4;
 constexpr int kResidentEpiThreads = 512;
 
@@ -839,6 +839,9 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS>(k, sm, c, ok);
         }
         stop = resident_grid_barrier(g.grid_sync + 1, abort_flag, stop);
+        // Every CTA of this grid is resident now (all have arrived at the barrier), so the kernels that follow may
+        // be scheduled beside it without taking an SM slot one of its CTAs still needs.
+        grid_dependency_launch_dependents();
         // ---- phase 1: density partials
         slot = 0;
         for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {

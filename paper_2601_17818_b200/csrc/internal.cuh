@@ -34,7 +34,15 @@ inline bool pdl_allowed(bool requested) { return requested && !kernel_timing_on(
 // ---- launchers (enqueue on `stream`, return VITCOP_OK or VITCOP_ERR_CUDA) -------------------------
 int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
                  int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
-                 cudaStream_t stream);
+                 cudaStream_t stream, bool late_wait = false);
+
+// K-norm to be enqueued in the middle of the filter's kernel chain (vitcop_collaborative_step): it does not depend
+// on the filter, so it runs beside the filter's sweep.
+struct KnormJob {
+    const void* K;
+    int B, H, N, d, vis_start, Nv;
+    float* score;
+};
 
 int launch_select(const float* score, const int32_t* label, int B, const int32_t* vis_len, int vis_len_uniform,
                   int Nv_cap, int mode, int largest, int budget, int32_t* keep_idx, int keep_stride,
@@ -49,7 +57,7 @@ size_t filter_workspace_bytes(int B, int n, int D);
 size_t similarity_workspace_bytes(int B, int n, int D);
 int launch_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params& p,
                   int n_centers, int32_t* label, int32_t* n_clusters, float* rho, float* delta2, int32_t* parent,
-                  void* workspace, cudaStream_t stream);
+                  void* workspace, cudaStream_t stream, const KnormJob* knorm = nullptr);
 int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, int row_begin, int row_end,
                            float* out, void* workspace, cudaStream_t stream);
 

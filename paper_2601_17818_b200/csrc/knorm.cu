@@ -38,8 +38,12 @@ __device__ __forceinline__ void sq_acc(const uint4& v, float& a0, float& a1) {
 template <int LPR, int UNROLL>
 __global__ void __launch_bounds__(kKnormThreads)
 knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh, int64_t sn, int vis_start,
-             const int32_t* __restrict__ vis_len, int vis_len_uniform, float* __restrict__ score, int Nv_cap) {
-    grid_dependency_wait();
+             const int32_t* __restrict__ vis_len, int vis_len_uniform, float* __restrict__ score, int Nv_cap,
+             int late_wait) {
+    // late_wait: K is known to be final already (the caller ordered its producer before the preceding grid), so
+    // this grid may run beside the preceding one; it still waits for it before it ends, which keeps "this grid
+    // has completed" meaning "everything before it has completed" for the kernels that follow.
+    if (!late_wait) grid_dependency_wait();
     const int b = blockIdx.y;
     const int nv = vis_len ? vis_len[b] : vis_len_uniform;
     constexpr int kTok = kKnormThreads / LPR;
@@ -79,13 +83,14 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
     // Only now may the next kernel's CTAs be scheduled: released earlier they would sit on the SMs waiting for
     // this grid while its own remaining CTAs queue behind them.
     grid_dependency_launch_dependents();
+    if (late_wait) grid_dependency_wait();
 }
 
 }  // namespace
 
 int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
                  int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
-                 cudaStream_t stream) {
+                 cudaStream_t stream, bool late_wait) {
     if (B <= 0 || Nv_cap <= 0 || H <= 0) return VITCOP_OK;
     const int d8 = d / 8;
     const int span = vis_len ? Nv_cap : vis_len_uniform;
@@ -106,7 +111,7 @@ int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t s
         cfg.numAttrs = pdl_allowed(true) ? 1 : 0;
         KernelTimeScope timed("knorm_kernel", stream);
         rc = record_cuda(cudaLaunchKernelEx(&cfg, kern, Kp, H, d8, sb, sh, sn, vis_start, vis_len, vis_len_uniform,
-                                            score, Nv_cap));
+                                            score, Nv_cap, late_wait ? 1 : 0));
     };
     if (d8 >= 16) go(knorm_kernel<16, 8>, 16);
     else if (d8 >= 8) go(knorm_kernel<8, 8>, 8);

@@ -398,3 +398,51 @@ def test_filter_then_quota_step_end_to_end():
     g = gpu_filter(f, p, 0, w.d_c, w.tau, w.n_centers)
     stats = _run_chain(w, use_labels=g.label)
     assert stats["steps"] == len(w.budgets)
+
+
+# ======================================================================================= Stage II in one call
+@pytest.mark.parametrize("name", ["tiny", "c0", "c1", "c2"])
+def test_collaborative_step_equals_filter_then_prune_step(name):
+    """vitcop_collaborative_step may reorder its kernels (the K-norm runs beside the clustering) but must return
+    exactly what vitcop_redundancy_filter followed by vitcop_prune_step returns; that pair is checked against the
+    oracle by the tests above."""
+    w = W.workload(name)
+    B, n = w.B, w.Nv
+    feat, pos = vb.bf16_tensor(W.make_features(w)), torch.from_numpy(W.make_positions(w).copy()).to(DEV)
+    K_b, V_b = W.make_kv(w, 0, n)
+    tK, tV, th = vb.bf16_tensor(K_b), vb.bf16_tensor(V_b), vb.bf16_tensor(W.make_hidden(w))
+    budget = w.budgets[0]
+    Ncap = w.T + budget
+
+    def outputs():
+        z = lambda *s, dt: torch.zeros(s, dtype=dt, device=DEV)
+        return dict(ho=z(B, Ncap, w.Dh, dt=torch.bfloat16), Ko=z(B, w.H, Ncap, w.d, dt=torch.bfloat16),
+                    Vo=z(B, w.H, Ncap, w.d, dt=torch.bfloat16), olen=z(B, dt=torch.int32),
+                    kpos=z(B, Ncap, dt=torch.int32), score=z(B, n, dt=torch.float32), kidx=z(B, n, dt=torch.int32),
+                    nkeep=z(B, dt=torch.int32), label=z(B, n, dt=torch.int32), ncl=z(B, dt=torch.int32))
+
+    ref = outputs()
+    ws_f = vb.alloc_workspace(vb.OP_FILTER, B=B, Nv=n, D=w.D)
+    ws_s = vb.alloc_workspace(vb.OP_PRUNE_STEP, B=B, Nv=n)
+    vb.vitcop_redundancy_filter(feat, pos, ref["label"], ref["ncl"], ws_f, metric=0, d_c=w.d_c, tau=w.tau,
+                                n_centers=w.n_centers)
+    vb.vitcop_prune_step(th, tK, tV, w.vis_start, n, n, budget, ref["ho"], ref["Ko"], ref["Vo"], ref["olen"], ws_s,
+                         label=ref["label"], kept_pos=ref["kpos"], score_out=ref["score"], keep_idx_out=ref["kidx"],
+                         n_keep_out=ref["nkeep"])
+    assert vb.vitcop_poll_status(ws_f) == vb.OK and vb.vitcop_poll_status(ws_s) == vb.OK
+    for rep in range(2):                                   # twice: the second call runs on a used workspace
+        got = outputs()
+        ws = vb.alloc_workspace(vb.OP_COLLAB_STEP, B=B, Nv=n, D=w.D) if rep == 0 else ws
+        vb.vitcop_collaborative_step(feat, pos, th, tK, tV, w.vis_start, budget, got["ho"], got["Ko"], got["Vo"],
+                                     got["olen"], got["label"], got["ncl"], ws, metric=0, d_c=w.d_c, tau=w.tau,
+                                     n_centers=w.n_centers, kept_pos=got["kpos"], score_out=got["score"],
+                                     keep_idx_out=got["kidx"], n_keep_out=got["nkeep"])
+        assert vb.vitcop_poll_status(ws) == vb.OK
+        nk = ref["nkeep"].cpu().numpy()
+        assert nk.min() > 0
+        for key in ("label", "ncl", "score", "nkeep", "olen", "kpos"):
+            assert torch.equal(got[key], ref[key]), key
+        for b in range(B):
+            assert torch.equal(got["kidx"][b, : nk[b]], ref["kidx"][b, : nk[b]])
+        for key in ("ho", "Ko", "Vo"):
+            assert torch.equal(got[key].view(torch.int16), ref[key].view(torch.int16)), key
