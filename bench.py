@@ -63,7 +63,8 @@ def source_sha(name: str) -> str:
 def config_of(w, **extra):
     c = {"workload": w.name, "B": w.B, "Nv": w.Nv, "T": w.T, "H": w.H, "d": w.d, "D": w.D, "Dh": w.Dh,
          "budget": w.budgets[0], "n_centers": w.n_centers, "d_c": w.d_c, "tau": w.tau,
-         "mode": "redundancy filter (cosine) + fused prune step in cluster-quota mode"}
+         "mode": "Stage II in one call (vitcop_collaborative_step): redundancy filter (cosine), K-norm, cluster-quota "
+                 "selection, compaction"}
     c.update(extra)
     return c
 
@@ -205,6 +206,7 @@ class Step:
         self.kpos = e(B, self.Ncap, dt=torch.int32)
         self.ws_f = vb.alloc_workspace(vb.OP_FILTER, device=dev, B=B, Nv=n, D=w.D)
         self.ws_s = vb.alloc_workspace(vb.OP_PRUNE_STEP, device=dev, B=B, Nv=n)
+        self.ws_c = vb.alloc_workspace(vb.OP_COLLAB_STEP, device=dev, B=B, Nv=n, D=w.D)
 
     def upload(self, host, non_blocking=True):
         for name in ("feat", "pos", "K", "V", "hidden"):
@@ -222,6 +224,14 @@ class Step:
                                   n_keep_out=self.nkeep)
 
     def run(self):
+        """The whole hot path through the one-call Stage II entry point (same results as filter() + prune())."""
+        w = self.w
+        self.vb.vitcop_collaborative_step(self.feat, self.pos, self.hidden, self.K, self.V, w.vis_start, self.budget,
+                                          self.ho, self.Ko, self.Vo, self.olen, self.label, self.ncl, self.ws_c,
+                                          metric=0, d_c=w.d_c, tau=w.tau, n_centers=w.n_centers, kept_pos=self.kpos,
+                                          n_keep_out=self.nkeep)
+
+    def run_two_calls(self):
         self.filter()
         self.prune()
 
@@ -237,14 +247,16 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
     latency-bound; they are reported in microseconds only.
     """
     rows_out = w.B * w.T + nk_total
+    sweep = w.B * w.Nv * (w.Nv + 1) * w.D
     algo = {
+        "gram_resident_kernel": ("tensor", sweep),      # one pass over the symmetric half serves norms, Eq. 2 and Eq. 3
         "knorm_kernel": ("hbm", w.B * w.H * w.Nv * w.d * 2 + w.B * w.Nv * 4),
         "compact_kernel": ("hbm", 2 * rows_out * (w.Dh + 2 * w.H * w.d) * 2 + rows_out * 4 + w.B * 12 + nk_total * 4),
         "gram_tc_kernel<rho>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
         "gram_tc_kernel<delta>": ("tensor", w.B * w.Nv * (w.Nv + 1) * w.D),
     }
     src = {"knorm_kernel": "knorm.cu", "compact_kernel": "compact.cu", "gram_tc_kernel<rho>": "gram.cu",
-           "gram_tc_kernel<delta>": "gram.cu"}
+           "gram_tc_kernel<delta>": "gram.cu", "gram_resident_kernel": "gram.cu"}
     out = {}
     for name, (launches, ms) in per_kernel.items():
         us = ms * 1e3 / max(launches, 1)
@@ -374,6 +386,7 @@ def run_ours(args):
     kidx = torch.empty((w.B, w.Nv), dtype=torch.int32, device=dev)
     ws_sel = vb.alloc_workspace(vb.OP_SELECT, device=dev, B=w.B, Nv=w.Nv)
     stage_fns = {
+        "filter_then_prune_step": st.run_two_calls,
         "filter": st.filter,
         "knorm": lambda: vb.vitcop_knorm_score(st.K, w.vis_start, w.Nv, score),
         "select": lambda: vb.vitcop_select(score, w.Nv, st.budget, kidx, st.nkeep, ws_sel, label=st.label),

@@ -334,15 +334,6 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
         if (rc != VITCOP_OK) return rc;
     }
 
-    if (knorm) {
-        // The sweep before this point has released its dependents early: the K-norm streams K from HBM while the
-        // sweep's tensor-core and epilogue work goes on, and waits for the sweep before it ends.
-        rc = launch_knorm(knorm->K, knorm->B, knorm->H, knorm->d, (int64_t)knorm->H * knorm->N * knorm->d,
-                          (int64_t)knorm->N * knorm->d, knorm->d, knorm->vis_start, nullptr, knorm->Nv, knorm->score,
-                          knorm->Nv, stream, true);
-        if (rc != VITCOP_OK) return rc;
-    }
-
     const int nc = n_centers < n ? n_centers : n;
     const size_t smem = (size_t)n * 8 + (((size_t)n + 15) & ~(size_t)15) + (size_t)(nc > 0 ? nc : 1) * 4 + 16;
     if (smem > 48 * 1024) {
@@ -352,10 +343,23 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     pdl_config(cfg, attr, dim3(B), dim3(kFinThreads), smem, stream, true);
-    KernelTimeScope timed("vic_finalize_kernel", stream);
-    return record_cuda(cudaLaunchKernelEx(&cfg, vic_finalize_kernel, static_cast<const uint16_t*>(feat), n, D, nc,
-                                          (const float*)rho, (const unsigned long long*)best, (const float*)w,
-                                          (const float*)a, label, n_clusters, delta2_user, parent_user));
+    {
+        KernelTimeScope timed("vic_finalize_kernel", stream);
+        rc = record_cuda(cudaLaunchKernelEx(&cfg, vic_finalize_kernel, static_cast<const uint16_t*>(feat), n, D, nc,
+                                            (const float*)rho, (const unsigned long long*)best, (const float*)w,
+                                            (const float*)a, label, n_clusters, delta2_user, parent_user));
+        if (rc != VITCOP_OK) return rc;
+    }
+    if (knorm) {
+        // vic_finalize_kernel runs one CTA per sample and releases its dependents when it starts: the K-norm, which
+        // does not depend on the clustering, streams K from HBM on the other SMs meanwhile and waits for the
+        // finalize kernel before it ends.  (Beside the Gram sweep it would not fit: that kernel's CTAs hold most
+        // of each SM's registers.)
+        rc = launch_knorm(knorm->K, knorm->B, knorm->H, knorm->d, (int64_t)knorm->H * knorm->N * knorm->d,
+                          (int64_t)knorm->N * knorm->d, knorm->d, knorm->vis_start, nullptr, knorm->Nv, knorm->score,
+                          knorm->Nv, stream, true);
+    }
+    return rc;
 }
 
 int launch_similarity_rows(const void* feat, int B, int n, int D, int metric, int row_begin, int row_end, float* out,
