@@ -315,6 +315,10 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
         g.rho_out = rho;
         g.rho_user = rho_user;
         g.grid_sync = reinterpret_cast<unsigned int*>(ws) + 2;       // zeroed with the status word at the start of the call
+        if (knorm) {                                                 // computed by the sweep's waiting epilogue warps
+            g.kn_K = knorm->K; g.kn_score = knorm->score;
+            g.kn_H = knorm->H; g.kn_N = knorm->N; g.kn_d = knorm->d; g.kn_vis_start = knorm->vis_start; g.kn_Nv = knorm->Nv;
+        }
         rc = launch_gram_resident(feat, g, make_gram_tiling(n, 128), stream);
         if (rc != VITCOP_OK) return rc;
     } else {
@@ -350,7 +354,7 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
                                             (const float*)a, label, n_clusters, delta2_user, parent_user));
         if (rc != VITCOP_OK) return rc;
     }
-    if (knorm) {
+    if (knorm && !resident) {
         // vic_finalize_kernel runs one CTA per sample and releases its dependents when it starts: the K-norm, which
         // does not depend on the clustering, streams K from HBM on the other SMs meanwhile and waits for the
         // finalize kernel before it ends.  (Beside the Gram sweep it would not fit: that kernel's CTAs hold most

@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include "gram.cuh"
+#include "knorm.cuh"
 
 namespace vitcop {
 namespace {
@@ -824,6 +825,29 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         bool stop = false;
         grid_dependency_wait();
 
+        // ---- while the tensor cores fill the accumulators: the K-norm of the step (Eq. 4), if the caller has one.
+        //      It streams K from HBM, which the Gram tiles (fed from L2) leave idle.  16 lanes per token.
+        if (g.kn_K) {
+            const int d8 = g.kn_d / 8;
+            const int64_t sn = d8, sh = (int64_t)g.kn_N * d8, sb = (int64_t)g.kn_H * sh;
+            const uint4* Kp = static_cast<const uint4*>(g.kn_K);
+            const int sub = e & 15;
+            const long long tokens = (long long)g.B * g.kn_Nv;
+            // a warp serves two consecutive tokens; the loop runs on the warp's first token so that all 32 lanes
+            // stay together for the shuffles
+            for (long long tw = (long long)blockIdx.x * (kResidentEpiThreads / 16) + 2 * (e >> 5); tw < tokens;
+                 tw += (long long)gridDim.x * (kResidentEpiThreads / 16)) {
+                const long long tk = tw + ((e >> 4) & 1);
+                const bool live = tk < tokens;
+                const int b = live ? (int)(tk / g.kn_Nv) : 0, i = live ? (int)(tk - (long long)b * g.kn_Nv) : 0;
+                float part = 0.f;
+                if (live)
+                    part = knorm_token_partial<16, 8>(Kp + b * sb + (int64_t)(g.kn_vis_start + i) * sn, g.kn_H, d8, sh, sub);
+#pragma unroll
+                for (int off = 8; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                if (live && sub == 0) g.kn_score[(size_t)b * g.kn_Nv + i] = sqrtf(part);
+            }
+        }
         // ---- phase 0: the diagonal tiles give g_ii, hence the per-token factors every other epilogue needs
         uint32_t slot = 0;
         for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {

@@ -57,6 +57,11 @@ struct GramArgs {
     float* rho_out;             // [B, n] written by the resident sweep (same memory as rho)
     float* rho_user;            // [B, n] optional copy of rho for the caller
     unsigned int* grid_sync;    // two zeroed counters for the resident sweep's grid-wide barriers
+    // Optional K-norm (Eq. 4) for the resident sweep's epilogue warps to compute while the tensor cores fill the
+    // accumulators: K bf16 [B, kn_H, kn_N, kn_d] dense, span [kn_vis_start, kn_vis_start + kn_Nv), score [B, kn_Nv].
+    const void* kn_K;
+    float* kn_score;
+    int kn_H, kn_N, kn_d, kn_vis_start, kn_Nv;
     int* status;                // device status word
 };
 

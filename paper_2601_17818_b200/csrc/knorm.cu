@@ -5,36 +5,14 @@
 // product is exact in fp32), accumulates over heads in registers and the group finishes with
 // xor-shuffles.  Consecutive tokens of one head are contiguous in memory, so a CTA's loads of one
 // head form one contiguous run of TOKENS_PER_CTA * d * 2 bytes.
-#include "internal.cuh"
+#include "knorm.cuh"
 
 namespace vitcop {
 namespace {
 
 constexpr int kKnormThreads = 128;
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-    uint4 v;
-    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ void sq_acc(const uint4& v, float& a0, float& a1) {
-    float x;
-    x = bf16lo(v.x); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.x); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.y); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.y); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.z); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.z); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.w); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.w); a1 = fmaf(x, x, a1);
-}
-
 // Strides are in units of 16 bytes (8 elements).
-// The loads of head batch k + 1 are issued before the squares of batch k are accumulated, so that every
-// thread always has UNROLL 16-byte requests in flight and the batches do not run in lock step.
 template <int LPR, int UNROLL>
 __global__ void __launch_bounds__(kKnormThreads)
 knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh, int64_t sn, int vis_start,
@@ -49,34 +27,9 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
     constexpr int kTok = kKnormThreads / LPR;
     const int sub = threadIdx.x % LPR;
     const int i = blockIdx.x * kTok + threadIdx.x / LPR;
-    float a0 = 0.f, a1 = 0.f;
-    if (i < nv) {
-        const uint4* base = K + b * sb + (int64_t)(vis_start + i) * sn;
-        for (int c = sub; c < d8; c += LPR) {
-            const uint4* p = base + c;
-            const int full = H / UNROLL * UNROLL;
-            if (full > 0) {
-                uint4 cur[UNROLL], nxt[UNROLL];
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) cur[u] = ld_stream(p + (int64_t)u * sh);
-                for (int h = UNROLL; h < full; h += UNROLL) {
-#pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) nxt[u] = ld_stream(p + (int64_t)(h + u) * sh);
-#pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) sq_acc(cur[u], a0, a1);
-#pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) cur[u] = nxt[u];
-                }
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) sq_acc(cur[u], a0, a1);
-            }
-            for (int h = full; h < H; ++h) {
-                const uint4 v = ld_stream(p + (int64_t)h * sh);
-                sq_acc(v, a0, a1);
-            }
-        }
-    }
-    float acc = a0 + a1;
+    float acc = 0.f;
+    if (i < nv)
+        acc = knorm_token_partial<LPR, UNROLL>(K + b * sb + (int64_t)(vis_start + i) * sn, H, d8, sh, sub);
 #pragma unroll
     for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (i < nv && sub == 0) score[(int64_t)b * Nv_cap + i] = sqrtf(acc);
