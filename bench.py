@@ -38,10 +38,9 @@ UNIT = "tokens/s"
 # (bytes per launch on the bench workload, sha1 of the kernel's source file when the counters were taken).
 # A kernel whose source changed since reports traffic null.
 NCU_TRAFFIC = {
-    "gram_tc_kernel<delta>": (19137024, "602bd8329f76"),
-    "gram_tc_kernel<rho>": (18940416, "602bd8329f76"),
-    "knorm_kernel": (75522560 + 1190400, "3e4bfc525f97"),
-    "compact_kernel": (33737728 + 1013760, "619ac324b74f"),
+    "gram_resident_kernel": (94523904 + 3087360, "42ee52f3e8bd"),
+    "knorm_kernel": (75522560 + 1326848, "6accb3df2988"),
+    "compact_kernel": (33764864 + 976896, "619ac324b74f"),
 }
 
 
