@@ -322,11 +322,8 @@ def run_ours(args):
     st.upload(host, non_blocking=False)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)     # > 4x the 126 MB L2
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    from paper_2601_17818_b200 import replicas
+    barrier = replicas.barrier
 
     def timed(fn, steps, warmup):
         """Per-step CUDA-event times (ms) with an L2 flush before every step."""
@@ -344,11 +341,7 @@ def run_ours(args):
         return np.array([a.elapsed_time(b) for a, b in evs], dtype=np.float64)
 
     def max_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return x
+        return replicas.max_over_ranks(x, dev)
 
     # whole step, device resident ------------------------------------------------------------------------
     sampler = ClockSampler(local)
@@ -359,7 +352,7 @@ def run_ours(args):
     nk_total = int(n_keep.sum())
     pruned_per_step = int((w.Nv - n_keep).sum())
     total_ms = max_over_ranks(float(t_step.sum()))
-    value = world * pruned_per_step * args.steps / (total_ms * 1e-3)
+    value = replicas.whole_job_rate(pruned_per_step, args.steps, float(t_step.sum()), dev)
 
     # per-kernel device times: the library brackets each of its kernels with CUDA events on the stream ----
     n_kt = max(10, min(args.steps, 50))

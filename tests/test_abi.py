@@ -100,6 +100,31 @@ def test_argument_validation_happens_on_the_host(L):
     assert L.vitcop_prune_step(null, a, null, 1, 1, 8, 8, 8, null, 0, null, 4, 4, null, 2, null, b, null, 8, null, fake, null, null, null, null, 0, null) == vb.ERR_WORKSPACE
 
 
+def test_argument_validation_of_the_wider_entry_points(L):
+    fake, odd, ws, null = C.c_void_p(0x1000), C.c_void_p(0x1008), C.c_void_p(0x10000), None
+    a, b = C.c_void_p(0x100000), C.c_void_p(0x900000)
+    fp = vb.FilterParams(0, 0.5, 0.6, 0.05, 0)
+    # merge: required pointers, Dh % 8, workspace
+    assert L.vitcop_merge_clusters(null, 1, 8, 8, 0, null, 4, 4, fake, fake, null, null, fake, fake, fake, 4, ws, 1 << 20, null) == vb.ERR_INVALID_ARG
+    assert L.vitcop_merge_clusters(a, 1, 8, 12, 0, null, 4, 4, fake, fake, null, null, fake, fake, fake, 4, ws, 1 << 20, null) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_merge_clusters(a, 1, 8, 8, 6, null, 4, 4, fake, fake, null, null, fake, fake, fake, 4, ws, 1 << 20, null) == vb.ERR_INVALID_ARG   # span > N
+    assert L.vitcop_merge_clusters(a, 1, 8, 8, 0, null, 4, 4, fake, fake, null, null, fake, fake, fake, 4, ws, 8, null) == vb.ERR_WORKSPACE
+    # saliency
+    assert L.vitcop_cls_saliency(null, fake, 1, 1, 4, 8, 0.5, fake, null, ws, 1 << 20, null) == vb.ERR_INVALID_ARG
+    assert L.vitcop_cls_saliency(fake, fake, 1, 1, 4, 12, 0.5, fake, null, ws, 1 << 20, null) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_cls_saliency(fake, odd, 1, 1, 4, 8, 0.5, fake, null, ws, 1 << 20, null) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_cls_saliency(fake, fake, 1, 1, 4, 8, 0.5, fake, null, ws, 16, null) == vb.ERR_WORKSPACE
+    # one-call Stage II: needs labels out, a valid metric / cutoff, D % 64, a workspace
+    args = lambda feat=fake, D=64, f=fp, lab=fake, wsb=1 << 24: (feat, null, D, C.byref(f), null, a, null, 1, 1, 8, 8, 8, 0, 4, 2, null, b, null, 8, null, fake, lab, fake, null, null, null, ws, wsb, null)
+    assert L.vitcop_collaborative_step(*args(lab=null)) == vb.ERR_INVALID_ARG
+    assert L.vitcop_collaborative_step(*args(f=vb.FilterParams(0, 0.0, 0.6, 0.05, 0))) == vb.ERR_INVALID_ARG
+    assert L.vitcop_collaborative_step(*args(D=72)) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_collaborative_step(*args(wsb=64)) == vb.ERR_WORKSPACE
+    assert vb.vitcop_workspace_bytes(vb.OP_COLLAB_STEP, B=2, Nv=100, D=64) > vb.vitcop_workspace_bytes(vb.OP_FILTER, B=2, Nv=100, D=64)
+    assert vb.vitcop_workspace_bytes(vb.OP_MERGE, B=2, Nv=100, N=10) >= 256 + 2 * 100 * 2
+    assert vb.vitcop_workspace_bytes(vb.OP_SALIENCY, B=2, H=4, N=33) >= 2 * 4 * 33 * 4
+
+
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(vb, "_lib", None)
     monkeypatch.setattr(vb, "LIB_PATH", str(tmp_path / "nope.so"))
