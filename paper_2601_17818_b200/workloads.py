@@ -261,13 +261,19 @@ def make_scores(seed: int, B: int, n: int, kind: str = "lognormal") -> np.ndarra
     raise ValueError(kind)
 
 
-def make_labels(seed: int, B: int, n: int, n_clusters: int) -> np.ndarray:
-    """int32 [B, n] random cluster labels; a label is the token index of its cluster's centre."""
+def make_labels(seed: int, B: int, n: int, n_clusters: int, skew: float = 0.0) -> np.ndarray:
+    """int32 [B, n] random cluster labels; a label is the token index of its cluster's centre.
+
+    Cluster sizes are multinomial-even by default; ``skew`` in (0, 1) first hands that share of the tokens to one
+    cluster (a large background cluster beside many small ones)."""
     rng = _rng(seed, 32, 8, n)
     out = np.empty((B, n), dtype=np.int32)
     for b in range(B):
         centres = np.sort(rng.permutation(n)[:n_clusters]).astype(np.int32)
         lab = centres[rng.integers(0, n_clusters, size=n)]
+        if skew > 0.0:
+            big = centres[int(rng.integers(0, n_clusters))]
+            lab[rng.random(n) < skew] = big
         lab[centres] = centres                                  # a centre carries its own index
         out[b] = lab
     return out

@@ -101,18 +101,25 @@ def test_select_ragged_lengths():
         assert np.all(mask[b, vl[b]:] == 7)               # mask past the span is untouched
 
 
+# Even cluster sizes take the per-cluster rank search; a dominant cluster (skew) takes the sort below 4096 tokens and
+# the per-cluster radix search above; more than 1024 clusters always take the sort.
 @pytest.mark.parametrize("kind", ["lognormal", "ties", "equal"])
-def test_select_quota_exact(kind):
-    for n, ncl in [(1, 1), (10, 2), (97, 7), (576, 29), (1000, 1000), (2880, 144), (16384, 820)]:
+@pytest.mark.parametrize("skew", [0.0, 0.7])
+def test_select_quota_exact(kind, skew):
+    cases = [(1, 1), (10, 2), (97, 7), (576, 29), (1000, 1000), (2880, 144), (16384, 820),
+             (4097, 3), (5000, 40), (6000, 1024), (8192, 2000)]
+    if skew:
+        cases = [(97, 7), (576, 29), (2880, 144), (4097, 3), (5000, 40), (6000, 1024), (16384, 820), (16384, 2)]
+    for n, ncl in cases:
         score = W.make_scores(n + 1, 2, n, kind)
-        label = W.make_labels(n, 2, n, ncl)
+        label = W.make_labels(n, 2, n, ncl, skew=skew)
         for budget in sorted({ncl, ncl + 1, (n + ncl) // 2, n}):
             keeps, nk, mask, status = gpu_select(score, budget, label=label)
             assert status == vb.OK
             for b in range(2):
                 want, nc, _ = oracle.select_quota(score[b].astype(np.float64), label[b], budget)
                 assert nc == ncl
-                assert np.array_equal(keeps[b], want), (n, ncl, budget, kind)
+                assert np.array_equal(keeps[b], want), (n, ncl, budget, kind, skew)
                 assert nk[b] + nc <= budget
         if ncl > 1:                                        # budget below the cluster count: device-side status
             keeps, nk, _, status = gpu_select(score, ncl - 1, label=label)
