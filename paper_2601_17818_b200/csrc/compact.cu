@@ -56,16 +56,34 @@ compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, co
                int keep_stride, const int32_t* __restrict__ n_keep, uint4* __restrict__ hidden_out,
                uint4* __restrict__ K_out, uint4* __restrict__ V_out, int Ncap, int32_t* __restrict__ kept_pos,
                int32_t* __restrict__ out_len) {
-    grid_dependency_wait();
     const int b = blockIdx.y;
     const int r = blockIdx.x;
     const int L = seq_len ? min(seq_len[b], N) : N;
+    const int64_t head_in = (int64_t)N * d8, head_out = (int64_t)Ncap * d8;
+    // A row in front of the visual span keeps its place whatever the selection turns out to be: it is copied
+    // before this kernel waits for the selection, while the kernels that produce it are still running.  (The
+    // tensors copied here are inputs of the whole call, complete before its first kernel started.)
+    const bool prefix_row = r < min(vis_start, L) && r < Ncap;
+    if (prefix_row) {
+        if (hidden)
+            copy_segments(hidden + ((int64_t)b * N + r) * dh8, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8, dh8, 0,
+                          0, 31);
+        if (K)
+            copy_segments(K + ((int64_t)b * H * N + r) * d8, K_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
+                          head_in, head_out, d8_shift);
+        if (V)
+            copy_segments(V + ((int64_t)b * H * N + r) * d8, V_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
+                          head_in, head_out, d8_shift);
+        if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = r;
+        if (r != 0) return;                                // row 0 still reports the sample's new length
+    }
+    grid_dependency_wait();
     int nv = vis_len ? vis_len[b] : vis_len_uniform;
     nv = max(0, min(nv, L - vis_start));
     const int nk = max(0, min(n_keep[b], nv));
     const int olen = L - nv + nk;
     if (r == 0 && threadIdx.x == 0) out_len[b] = olen;
-    if (r >= Ncap) return;
+    if (r >= Ncap || prefix_row) return;
     if (r >= olen) {
         if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = -1;
         return;
@@ -82,7 +100,6 @@ compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, co
     if (hidden)
         copy_segments(hidden + ((int64_t)b * N + src_row) * dh8, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8, dh8, 0,
                       0, 31);
-    const int64_t head_in = (int64_t)N * d8, head_out = (int64_t)Ncap * d8;
     if (K)
         copy_segments(K + ((int64_t)b * H * N + src_row) * d8, K_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
                       head_in, head_out, d8_shift);

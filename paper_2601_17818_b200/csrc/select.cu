@@ -23,6 +23,9 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     __shared__ uint32_t warp_sums[kSelWarps];
     __shared__ uint32_t s_digit, s_krem, s_whole;
 
+    // The compaction that follows may start at once: it copies the rows that do not depend on the selection and
+    // waits for this kernel to complete before it reads the kept indices.
+    grid_dependency_launch_dependents();
     grid_dependency_wait();
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -116,7 +119,6 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
         kept = keep_running;
     }
     if (tid == 0) n_keep[b] = (int32_t)kept;
-    grid_dependency_launch_dependents();
 }
 
 // ------------------------------------------------------------------------------------------ quota
@@ -125,10 +127,10 @@ select_quota_kernel(const float* __restrict__ score, const int32_t* __restrict__
                     const int32_t* __restrict__ vis_len, int vis_len_uniform, int Nv_cap, int P_cap, int budget,
                     int32_t* __restrict__ keep_idx, int keep_stride, int32_t* __restrict__ n_keep,
                     uint8_t* __restrict__ keep_mask, int* __restrict__ status_word) {
+    grid_dependency_launch_dependents();                  // see select_plain_kernel
     grid_dependency_wait();
     select_quota_body(score, label, vis_len, vis_len_uniform, Nv_cap, P_cap, budget, keep_idx, keep_stride, n_keep,
                       keep_mask, status_word, blockIdx.x);
-    grid_dependency_launch_dependents();
 }
 
 }  // namespace
