@@ -117,7 +117,7 @@ typedef struct {
 } vitcop_filter_params;
 
 /*   feat       bf16 [B, n, D]          token features (D multiple of 64, n <= VITCOP_MAX_VISUAL_TOKENS)
- *   pos        fp32 [B, n, 2] or NULL  token coordinates; NULL disables the spatial test
+ *   pos        fp32 [B, n, 2] or NULL  token coordinates (8-byte aligned); NULL disables the spatial test
  *   p          host pointer
  *   label      int32 [B, n]   out      token index of the centre of each token's cluster
  *   n_clusters int32 [B]      out      number of centres (same for every sample)

@@ -55,6 +55,7 @@ KernelTimeScope::~KernelTimeScope() {
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
 inline bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
@@ -332,7 +333,7 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
     if (rc != VITCOP_OK) return rc;
     rc = check_span(N, vis_start, nullptr, Nv, Nv);
     if (rc != VITCOP_OK) return rc;
-    if (D % 64 || !aligned16(feat) || Nv > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
+    if (D % 64 || !aligned16(feat) || !aligned8(pos) || Nv > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
     const size_t filter_bytes = align_up(filter_workspace_bytes(B, Nv, D), 256);
     const StepWs lay(B, Nv);
     if (!workspace || workspace_bytes < filter_bytes + lay.total || !aligned256(workspace)) return VITCOP_ERR_WORKSPACE;
@@ -348,7 +349,7 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
     float* score = score_out ? score_out : reinterpret_cast<float*>(ws2 + lay.off_score);
     int32_t* keep = keep_idx_out ? keep_idx_out : reinterpret_cast<int32_t*>(ws2 + lay.off_keep);
     int32_t* nkeep = n_keep_out ? n_keep_out : reinterpret_cast<int32_t*>(ws2 + lay.off_nkeep);
-    rc = reset_status(workspace, s);
+    rc = record_cuda(cudaMemsetAsync(workspace, 0, filter_zeroed_bytes(B, Nv), s));
     if (rc != VITCOP_OK) return rc;
     if (B == 0) return VITCOP_OK;
     if (Nv > 0) {
@@ -417,7 +418,8 @@ int vitcop_redundancy_filter(const void* feat, const float* pos, int B, int n, i
     if (!feat || !p || !label || !n_clusters || B < 0 || n < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
     if (p->metric != 0 && p->metric != 1) return VITCOP_ERR_INVALID_ARG;
     if (!(p->d_c > 0.f)) return VITCOP_ERR_INVALID_ARG;
-    if (D % 64 || !aligned16(feat) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (D % 64 || !aligned16(feat) || !aligned8(pos) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535)
+        return VITCOP_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < filter_workspace_bytes(B, n, D) || !aligned256(workspace))
         return VITCOP_ERR_WORKSPACE;
     int nc = p->n_centers;
@@ -427,7 +429,7 @@ int vitcop_redundancy_filter(const void* feat, const float* pos, int B, int n, i
     }
     if (nc > n) nc = n;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int rc = reset_status(workspace, s);
+    int rc = record_cuda(cudaMemsetAsync(workspace, 0, filter_zeroed_bytes(B, n), s));
     if (rc != VITCOP_OK) return rc;
     if (B == 0 || n == 0) return VITCOP_OK;
     return launch_filter(feat, pos, B, n, D, *p, nc, label, n_clusters, rho, delta2, parent, workspace, s);
@@ -438,7 +440,8 @@ int vitcop_similarity_rows(const void* feat, int B, int n, int D, int metric, in
     if (!feat || !out || B < 0 || n < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
     if (metric != 0 && metric != 1) return VITCOP_ERR_INVALID_ARG;
     if (row_begin < 0 || row_end < row_begin || row_end > n) return VITCOP_ERR_INVALID_ARG;
-    if (D % 64 || !aligned16(feat) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (D % 64 || !aligned16(feat) || n > VITCOP_MAX_VISUAL_TOKENS || B > 65535)
+        return VITCOP_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < similarity_workspace_bytes(B, n, D) || !aligned256(workspace))
         return VITCOP_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -247,12 +247,15 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-// Workspace of the filter: status | w | a | rho | best | rho partials [B, slots, n_pad] (sized for either tile width)
+// Workspace of the filter: status block | row-block flags [B, ceil(n / 128)] | w | a | rho | best |
+// rho partials [B, slots, n_pad] (sized for either tile width).  The status block and the flags are zeroed at the
+// start of every call.  Words of the status block: 0 status, 2 grid barrier.
 struct FilterWs {
-    size_t off_w, off_a, off_rho, off_best, off_part, total;
+    size_t off_flags, off_w, off_a, off_rho, off_best, off_part, total;
     FilterWs(int B, int n) {
         size_t o = kStatusBytes;
         const size_t bn = (size_t)B * n;
+        off_flags = o; o += align_up((size_t)B * ((n + kGramBM - 1) / kGramBM) * 4, 256);
         off_w = o;    o += align_up(bn * 4, 256);
         off_a = o;    o += align_up(bn * 4, 256);
         off_rho = o;  o += align_up(bn * 4, 256);
@@ -277,6 +280,8 @@ void pdl_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 grid, d
 }
 
 }  // namespace
+
+size_t filter_zeroed_bytes(int B, int n) { return FilterWs(B, n).off_w; }
 
 size_t filter_workspace_bytes(int B, int n, int D) {
     (void)D;
@@ -310,14 +315,21 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     // The first kernel of the call is launched without programmatic overlap, so everything queued before the call
     // (the producer of the features included) has completed when it starts.
     int rc;
+    int knorm_in_sweep = 0;                                // leading samples whose K-norm the Gram sweep computes
     const bool resident = gram_fits_resident(B, n);
     if (resident) {
         g.rho_out = rho;
         g.rho_user = rho_user;
         g.grid_sync = reinterpret_cast<unsigned int*>(ws) + 2;       // zeroed with the status word at the start of the call
-        if (knorm) {                                                 // computed by the sweep's waiting epilogue warps
-            g.kn_K = knorm->K; g.kn_score = knorm->score;
-            g.kn_H = knorm->H; g.kn_N = knorm->N; g.kn_d = knorm->d; g.kn_vis_start = knorm->vis_start; g.kn_Nv = knorm->Nv;
+        g.diag_ready = reinterpret_cast<unsigned int*>(ws + l.off_flags);
+        if (knorm && gram_resident_takes_knorm(knorm->H, knorm->d)) {
+            // The sweep's two idle warps take the K-norm of the first samples, about as many as they finish while
+            // the epilogue warps work on the accumulators; the other samples follow beside vic_finalize_kernel.
+            knorm_in_sweep = (5 * knorm->B + 8) / 16;
+            if (knorm_in_sweep > 0) {
+                g.kn_K = knorm->K; g.kn_score = knorm->score; g.kn_B = knorm_in_sweep;
+                g.kn_H = knorm->H; g.kn_N = knorm->N; g.kn_d = knorm->d; g.kn_vis_start = knorm->vis_start; g.kn_Nv = knorm->Nv;
+            }
         }
         rc = launch_gram_resident(feat, g, make_gram_tiling(n, 128), stream);
         if (rc != VITCOP_OK) return rc;
@@ -354,13 +366,15 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
                                             (const float*)a, label, n_clusters, delta2_user, parent_user));
         if (rc != VITCOP_OK) return rc;
     }
-    if (knorm && !resident) {
+    if (knorm && knorm_in_sweep < knorm->B) {
         // vic_finalize_kernel runs one CTA per sample and releases its dependents when it starts: the K-norm, which
         // does not depend on the clustering, streams K from HBM on the other SMs meanwhile and waits for the
         // finalize kernel before it ends.  (Beside the Gram sweep it would not fit: that kernel's CTAs hold most
         // of each SM's registers.)
-        rc = launch_knorm(knorm->K, knorm->B, knorm->H, knorm->d, (int64_t)knorm->H * knorm->N * knorm->d,
-                          (int64_t)knorm->N * knorm->d, knorm->d, knorm->vis_start, nullptr, knorm->Nv, knorm->score,
+        const int64_t stride_b = (int64_t)knorm->H * knorm->N * knorm->d;
+        rc = launch_knorm(static_cast<const uint16_t*>(knorm->K) + (size_t)knorm_in_sweep * stride_b,
+                          knorm->B - knorm_in_sweep, knorm->H, knorm->d, stride_b, (int64_t)knorm->N * knorm->d, knorm->d,
+                          knorm->vis_start, nullptr, knorm->Nv, knorm->score + (size_t)knorm_in_sweep * knorm->Nv,
                           knorm->Nv, stream, true);
     }
     return rc;

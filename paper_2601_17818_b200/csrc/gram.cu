@@ -237,8 +237,8 @@ struct GemmSmem {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kTileBytes = kStages * kStageBytes;
     // per column of the tile: w, a, rho, x, y; column reduction scratch: 4 x value, 4 x index;
-    // row reduction scratch: 3 x value, 3 x index
-    static constexpr int kEpiBytes = (5 + 4 + 4) * BN * 4 + (3 + 3) * BM * 4;
+    // row reduction scratch: 3 x value, 3 x index; per row of the tile: w, a, rho, x, y
+    static constexpr int kEpiBytes = (5 + 4 + 4) * BN * 4 + (3 + 3 + 5) * BM * 4;
     static constexpr int kBarBytes = 256;
     static constexpr int kTotal = 1024 /*alignment slack*/ + kTileBytes + kEpiBytes + kBarBytes;
 };
@@ -251,6 +251,25 @@ constexpr float kInf = __builtin_huge_valf();
 struct EpiSmem {
     float *colw, *cola, *colrho, *colx, *coly, *colred, *rowred;
     int *colidx, *rowidx;
+    float *roww, *rowa, *rowrho, *rowx, *rowy;
+    // Carves the arrays out of GemmSmem<BN>::kEpiBytes bytes at `base`.
+    template <int BN>
+    __device__ __forceinline__ void carve(uint8_t* base) {
+        colw = reinterpret_cast<float*>(base);
+        cola = colw + BN;
+        colrho = cola + BN;
+        colx = colrho + BN;
+        coly = colx + BN;
+        colred = coly + BN;                                     // [4][BN]
+        colidx = reinterpret_cast<int*>(colred + 4 * BN);       // [4][BN]
+        rowred = reinterpret_cast<float*>(colidx + 4 * BN);     // [3][BM]
+        rowidx = reinterpret_cast<int*>(rowred + 3 * BM);       // [3][BM]
+        roww = reinterpret_cast<float*>(rowidx + 3 * BM);
+        rowa = roww + BM;
+        rowrho = rowa + BM;
+        rowx = rowrho + BM;
+        rowy = rowx + BM;
+    }
 };
 struct EpiCall {
     int b, ti, tj;                 // sample, row tile, column tile
@@ -285,45 +304,68 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
     const bool row_valid = SYM ? (i < g.n) : (i < g.row_end);
     const size_t bo = (size_t)b * g.n;
 
-    // ---- per-column and per-row constants
-    for (int ce = e; ce < BN && !DIAG; ce += kEpiThreads) {
-        const int j = J0 + ce;
-        const bool cv = j < g.n;
-        colw[ce] = cv ? g.w[bo + j] : 0.f;
-        if (METRIC == 1) cola[ce] = cv ? g.a[bo + j] : 0.f;
-        if (MODE == GRAM_DELTA) {
-            float rj = 0.f;
-            if (cv) {
-                if (call.rho_from_part) {
-                    rj = rho_from_partials(g.part + (size_t)b * k.t.slots() * k.t.n_pad + j, k.t, j);
-                    if (ti == tj) {                        // the diagonal tile of a row block publishes its tokens' rho
-                        g.rho_out[bo + j] = rj;
-                        if (g.rho_user) g.rho_user[bo + j] = rj;
+    // ---- per-column and per-row constants.  One item per thread where the tile allows it -- column factors,
+    //      column rho and position, row factors, row rho and position -- so that all the global loads of the tile
+    //      are in flight together: one round trip to L2 instead of one per group.
+    const float* part_b = (MODE == GRAM_DELTA && call.rho_from_part)
+                              ? g.part + (size_t)b * k.t.slots() * k.t.n_pad : nullptr;
+    for (int it = e; it < 2 * BN + 2 * BM && !DIAG; it += kEpiThreads) {
+        if (it < BN) {
+            const int ce = it, j = J0 + ce;
+            const bool cv = j < g.n;
+            // (L2 loads: another CTA may have written these factors after this SM last cached their line)
+            colw[ce] = cv ? __ldcg(g.w + bo + j) : 0.f;
+            if (METRIC == 1) cola[ce] = cv ? __ldcg(g.a + bo + j) : 0.f;
+        } else if (it < 2 * BN) {
+            if (MODE == GRAM_DELTA) {
+                const int ce = it - BN, j = J0 + ce;
+                const bool cv = j < g.n;
+                float rj = 0.f;
+                float2 pj = make_float2(0.f, 0.f);
+                if (cv) {
+                    if (SPATIAL) pj = *reinterpret_cast<const float2*>(g.pos + 2 * (bo + j));
+                    if (call.rho_from_part) {
+                        rj = rho_from_partials(part_b + j, k.t, j);
+                        if (ti == tj) {                        // the diagonal tile of a row block publishes its tokens' rho
+                            g.rho_out[bo + j] = rj;
+                            if (g.rho_user) g.rho_user[bo + j] = rj;
+                        }
+                    } else {
+                        rj = g.rho[bo + j];
                     }
-                } else {
-                    rj = g.rho[bo + j];
                 }
+                colrho[ce] = rj;
+                if (SPATIAL) { colx[ce] = pj.x; coly[ce] = pj.y; }
             }
-            colrho[ce] = rj;
-            if (SPATIAL) {
-                colx[ce] = cv ? g.pos[2 * (bo + j)] : 0.f;
-                coly[ce] = cv ? g.pos[2 * (bo + j) + 1] : 0.f;
+        } else if (it < 2 * BN + BM) {
+            const int r = it - 2 * BN, ir = I0 + r;
+            const bool rv = SYM ? (ir < g.n) : (ir < g.row_end);
+            sm.roww[r] = rv ? __ldcg(g.w + bo + ir) : 0.f;
+            if (METRIC == 1) sm.rowa[r] = rv ? __ldcg(g.a + bo + ir) : 0.f;
+        } else if (MODE == GRAM_DELTA) {
+            const int r = it - 2 * BN - BM, ir = I0 + r;
+            float rr = 0.f;
+            float2 pr = make_float2(0.f, 0.f);
+            if (ir < g.n) {
+                if (SPATIAL) pr = *reinterpret_cast<const float2*>(g.pos + 2 * (bo + ir));
+                rr = call.rho_from_part ? rho_from_partials(part_b + ir, k.t, ir) : g.rho[bo + ir];
             }
+            sm.rowrho[r] = rr;
+            if (SPATIAL) { sm.rowx[r] = pr.x; sm.rowy[r] = pr.y; }
         }
-    }
-    const float w_i = (row_valid && !DIAG) ? g.w[bo + i] : 0.f;
-    const float a_i = METRIC == 1 ? (row_valid ? g.a[bo + i] : 0.f) : 1.f;
-    const float m2w_i = -2.f * w_i;
-    float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
-    if (MODE == GRAM_DELTA && row_valid) {
-        rho_i = call.rho_from_part ? rho_from_partials(g.part + (size_t)b * k.t.slots() * k.t.n_pad + i, k.t, i)
-                                   : g.rho[bo + i];
-        if (SPATIAL) { x_i = g.pos[2 * (bo + i)]; y_i = g.pos[2 * (bo + i) + 1]; }
     }
     // every pair of the tile has i < j < n: no masking needed
     const bool full = SYM && (J0 >= I0 + BM) && (J0 + BN <= g.n);
 
     epi_bar_sync<kEpiThreads>();
+    const float w_i = DIAG ? 0.f : sm.roww[rl];
+    const float a_i = METRIC == 1 ? (DIAG ? 0.f : sm.rowa[rl]) : 1.f;
+    const float m2w_i = -2.f * w_i;
+    float rho_i = 0.f, x_i = 0.f, y_i = 0.f;
+    if (MODE == GRAM_DELTA) {
+        rho_i = sm.rowrho[rl];
+        if (SPATIAL) { x_i = sm.rowx[rl]; y_i = sm.rowy[rl]; }
+    }
     if (ok && call.wait_bar) ok = mbar_wait(call.wait_bar, call.wait_parity, call.abort_flag);
     ok = __all_sync(0xffffffffu, ok);
 
@@ -523,15 +565,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned for the 128B swizzle
     uint8_t* gen = smem_raw + (tiles - raw);
-    float* colw = reinterpret_cast<float*>(gen + S::kTileBytes);
-    float* cola = colw + BN;
-    float* colrho = cola + BN;
-    float* colx = colrho + BN;
-    float* coly = colx + BN;
-    float* colred = coly + BN;                                     // [4][BN]
-    int* colidx = reinterpret_cast<int*>(colred + 4 * BN);         // [4][BN]
-    float* rowred = reinterpret_cast<float*>(colidx + 4 * BN);     // [3][BM]
-    int* rowidx = reinterpret_cast<int*>(rowred + 3 * BM);         // [3][BM]
+    EpiSmem sm;
+    sm.template carve<BN>(gen + S::kTileBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
     // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], drain
     const uint32_t bar_full = smem_u32(bars);
@@ -641,9 +676,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ epilogue (warps 2 ..)
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        EpiSmem sm;
-        sm.colw = colw; sm.cola = cola; sm.colrho = colrho; sm.colx = colx; sm.coly = coly;
-        sm.colred = colred; sm.colidx = colidx; sm.rowred = rowred; sm.rowidx = rowidx;
 
         grid_dependency_wait();                            // w, a, rho, best come from the preceding kernels
 
@@ -675,14 +707,20 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // the resident kernel: density and delta from ONE pass over the Gram tiles (small problems)
 // ------------------------------------------------------------------------------------------------
 // Every CTA owns at most kResidentSlots tiles of 128 x 128 and keeps all their accumulators in tensor memory
-// (4 x 128 of the 512 columns).  Phases of the epilogue warps:
-//   0. the diagonal tiles yield g_ii -> per-token normalisation factors; grid-wide barrier
-//   1. density epilogue of every tile -> rho partials; grid-wide barrier
+// (4 x 128 of the 512 columns).  Tiles are numbered with the diagonal ones first, so that these are the first
+// accumulators to complete.  Phases of the epilogue warps:
+//   0. the diagonal tiles yield g_ii -> per-token normalisation factors, published behind one flag per row block
+//   1. density epilogue of every tile (after the flags of its row and column block) -> rho partials;
+//      grid-wide barrier
 //   2. delta epilogue of every tile, re-reading the accumulators; rho of the tile's rows and columns is summed
 //      from the partials on the way (the diagonal tiles publish it)
-// The grid (at most one CTA per SM) is launched cooperatively, so all CTAs are resident together; the barriers
-// are counters in global memory with a bounded wait.  Dependents are released after the first barrier, when every
-// CTA is known to be resident: released earlier, their CTAs could take SM slots that CTAs of this grid still need.
+// The grid (at most one CTA per SM) is launched cooperatively, so all CTAs are resident together; flags and barrier
+// are words in global memory with bounded waits.  No wait can form a cycle: a flag is raised by a CTA that has
+// waited for nothing but its own tensor-core work.
+// The load warp and the MMA warp are idle once the CTA's last MMA is issued, and so are, a little later, the
+// operand buffers and -- for the rest of the kernel, which is arithmetic on the accumulators -- the memory system:
+// if the caller has a K-norm (Eq. 4) to compute, these two warps stream K through the operand buffers with bulk
+// copies and reduce it there (resident_knorm).
 constexpr int kResidentSlots = 4;
 constexpr int kResidentEpiThreads = 512;
 
@@ -708,6 +746,145 @@ __device__ __forceinline__ bool resident_grid_barrier(unsigned int* counter, vol
     return stop;
 }
 
+// Raises a flag once every epilogue thread's global writes are visible device-wide.
+__device__ __forceinline__ void resident_publish(unsigned int* flag) {
+    __threadfence();
+    epi_bar_sync<kResidentEpiThreads>();
+    if (threadIdx.x == 64) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
+}
+
+// Waits (bounded) until both flags are up.  Returns true when the grid must give up.
+__device__ __forceinline__ bool resident_wait_flags(const unsigned int* fa, const unsigned int* fb,
+                                                    volatile int* abort_flag, bool aborted) {
+    if (threadIdx.x == 64 && !aborted) {
+        const unsigned long long t0 = global_ns();
+        while (ld_acquire_u32(fa) == 0u || ld_acquire_u32(fb) == 0u) {
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+        }
+    }
+    const bool stop = epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
+    __threadfence();
+    return stop;
+}
+
+// Tile t of the resident sweep: the B * TI diagonal tiles first, then the tiles above the diagonal, sample by
+// sample, column tile by column tile.
+__device__ __forceinline__ void decode_resident_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
+    const int TI = k.t.TI;
+    const long long n_diag = (long long)k.g.B * TI;
+    if (t < n_diag) {
+        b = (int)(t / TI);
+        ti = tj = (int)(t - (long long)b * TI);
+        return;
+    }
+    const int above = TI * (TI - 1) / 2;                   // > 0 here: with TI == 1 every tile is diagonal
+    const long long u = t - n_diag;
+    b = (int)(u / above);
+    const int r = (int)(u - (long long)b * above);
+    int q = (int)((sqrtf(8.f * (float)r + 1.f) - 1.f) * 0.5f);
+    while (q > 0 && q * (q + 1) / 2 > r) --q;
+    while ((q + 1) * (q + 2) / 2 <= r) ++q;
+    tj = q + 1;
+    ti = r - q * (q + 1) / 2;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+constexpr int kKnChunkTokens = 8;                          // tokens per chunk: 8 threads each
+constexpr int kKnBuffers = 3;
+
+// K-norm (Eq. 4) by the 64 threads of warps 0 and 1, after the CTA's last MMA has completed.  Chunks of eight
+// consecutive tokens of one sample are copied head by head (one contiguous run per head) into the operand
+// buffers, up to three chunks in flight; eight threads reduce one token, each standing in for lanes s and s + 8
+// of the sixteen-lane reduction of the stand-alone kernel, so that both give the same bits.
+__device__ __forceinline__ void resident_knorm(const GramArgs& g, const uint8_t* buf_gen, uint32_t buf_smem,
+                                               uint32_t buf_bytes, uint32_t bar_kn, uint32_t bar_last_mma,
+                                               volatile int* abort_flag) {
+    const int tid = threadIdx.x;                           // 0 .. 63
+    auto all_ok = [](bool ok) {
+        uint32_t out;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.eq.b32 p, %1, 0;\n\t"
+            "bar.red.or.pred q, 2, 64, p;\n\t"
+            "selp.u32 %0, 0, 1, q;\n\t}"
+            : "=r"(out) : "r"((uint32_t)ok) : "memory");
+        return out != 0;
+    };
+    // the tensor cores read the operand buffers until the last MMA completes
+    if (!all_ok(mbar_wait(bar_last_mma, 0, abort_flag))) return;
+
+    const int H = g.kn_H, d8 = g.kn_d / 8, Nv = g.kn_Nv;
+    const uint32_t row_bytes = (uint32_t)d8 * 16u;
+    const uint32_t head_bytes = kKnChunkTokens * row_bytes;         // one head of a chunk
+    const uint32_t chunk_bytes = (uint32_t)H * head_bytes;
+    const int nbuf = min(kKnBuffers, (int)(buf_bytes / chunk_bytes));   // >= 1 (gram_resident_takes_knorm)
+    const int chunks_per_b = (Nv + kKnChunkTokens - 1) / kKnChunkTokens;
+    const long long total = (long long)g.kn_B * chunks_per_b;
+    const uint8_t* Kb = static_cast<const uint8_t*>(g.kn_K);
+    const size_t head_stride = (size_t)g.kn_N * row_bytes;
+
+    auto issue = [&](long long c, int buf) {               // thread 0
+        const int b = (int)(c / chunks_per_b);
+        const int i0 = (int)(c - (long long)b * chunks_per_b) * kKnChunkTokens;
+        const int cnt = min(kKnChunkTokens, Nv - i0);
+        const uint32_t run = (uint32_t)cnt * row_bytes;
+        mbar_expect_tx(bar_kn + 8 * buf, (uint32_t)H * run);
+        const uint8_t* src = Kb + ((size_t)b * H * g.kn_N + (size_t)(g.kn_vis_start + i0)) * row_bytes;
+        const uint32_t dst = buf_smem + (uint32_t)buf * chunk_bytes;
+        for (int h = 0; h < H; ++h) bulk_load(dst + (uint32_t)h * head_bytes, src + (size_t)h * head_stride, run, bar_kn + 8 * buf);
+    };
+    long long issued = 0;                                  // chunks this CTA has requested (thread 0)
+    if (tid == 0)
+        for (; issued < nbuf && blockIdx.x + issued * gridDim.x < total; ++issued)
+            issue(blockIdx.x + issued * gridDim.x, (int)issued);
+
+    const int tk = tid >> 3, s = tid & 7;
+    long long it = 0;
+    bool ok = true;
+    for (long long c = blockIdx.x; c < total; c += gridDim.x, ++it) {
+        const int buf = (int)(it % nbuf);
+        ok = all_ok(mbar_wait(bar_kn + 8 * buf, (uint32_t)((it / nbuf) & 1), abort_flag));
+        if (!ok) break;
+        const int b = (int)(c / chunks_per_b);
+        const int i0 = (int)(c - (long long)b * chunks_per_b) * kKnChunkTokens;
+        const int cnt = min(kKnChunkTokens, Nv - i0);
+        const uint4* rows = reinterpret_cast<const uint4*>(buf_gen + (size_t)buf * chunk_bytes) + (size_t)tk * d8;
+        const int head16 = kKnChunkTokens * d8;            // uint4 per head of a chunk
+        float part = 0.f;
+        if (tk < cnt) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                float a0 = 0.f, a1 = 0.f;
+                for (int piece = s + 8 * q; piece < d8; piece += 16) {
+#pragma unroll 8
+                    for (int h = 0; h < H; ++h) knorm_sq_acc(rows[(size_t)h * head16 + piece], a0, a1);
+                }
+                part += a0 + a1;
+            }
+        }
+#pragma unroll
+        for (int off = 4; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+        if (tk < cnt && s == 0) g.kn_score[(size_t)b * Nv + i0 + tk] = sqrtf(part);
+        asm volatile("bar.sync 2, 64;" ::: "memory");      // the buffer has been read by everyone
+        if (tid == 0) {
+            const long long cn = blockIdx.x + issued * gridDim.x;
+            if (cn < total) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue(cn, buf);
+                ++issued;
+            }
+        }
+    }
+    if (!ok && tid == 0) {
+        // giving up: wait (bounded) for the copies still in flight before the CTA's shared memory goes away
+        for (long long j = it; j < issued; ++j) mbar_drain(bar_kn + 8 * (int)(j % nbuf), (uint32_t)((j / nbuf) & 1));
+    }
+}
+
 template <int METRIC, bool SPATIAL>
 __global__ void __launch_bounds__(64 + kResidentEpiThreads, 1)
 gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -721,22 +898,16 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (tiles - raw);
     EpiSmem sm;
-    sm.colw = reinterpret_cast<float*>(gen + S::kTileBytes);
-    sm.cola = sm.colw + BN;
-    sm.colrho = sm.cola + BN;
-    sm.colx = sm.colrho + BN;
-    sm.coly = sm.colx + BN;
-    sm.colred = sm.coly + BN;
-    sm.colidx = reinterpret_cast<int*>(sm.colred + 4 * BN);
-    sm.rowred = reinterpret_cast<float*>(sm.colidx + 4 * BN);
-    sm.rowidx = reinterpret_cast<int*>(sm.rowred + 3 * BM);
+    sm.template carve<BN>(gen + S::kTileBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
-    // barriers: full[kStages], empty[kStages], tmem_full[kResidentSlots], drain
+    // barriers: full[kStages], empty[kStages], tmem_full[kResidentSlots], drain, knorm[kKnBuffers]
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * S::kStages;
     const uint32_t bar_tfull = bar_empty + 8 * S::kStages;
     const uint32_t bar_drain = bar_tfull + 8 * kResidentSlots;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + kResidentSlots + 1);
+    const uint32_t bar_kn = bar_drain + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + kResidentSlots + 1 + kKnBuffers);
+    static_assert((2 * S::kStages + kResidentSlots + 1 + kKnBuffers) * 8 + 8 <= S::kBarBytes, "barrier block too small");
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -749,6 +920,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
         for (int a = 0; a < kResidentSlots; ++a) mbar_init(bar_tfull + 8 * a, 1);
         mbar_init(bar_drain, 1);
+        for (int a = 0; a < kKnBuffers; ++a) mbar_init(bar_kn + 8 * a, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
@@ -771,7 +943,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
                 int b, ti, tj;
-                decode_tile<BN, true, false>(k, t, b, ti, tj);
+                decode_resident_tile(k, t, b, ti, tj);
                 const int I0 = ti * BM, J0 = tj * BN;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -818,6 +990,14 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 mbar_drain(bar_drain, 0);
             }
         }
+    }
+    if (warp < 2) {
+        __syncwarp();
+        if (g.kn_K) {
+            const long long my_tiles = (total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;   // >= 1
+            resident_knorm(g, gen, tiles, (uint32_t)S::kTileBytes, bar_kn, bar_tfull + 8 * (uint32_t)(my_tiles - 1),
+                           abort_flag);
+        }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..17)
         const int e = threadIdx.x - 64;
@@ -825,34 +1005,11 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         bool stop = false;
         grid_dependency_wait();
 
-        // ---- while the tensor cores fill the accumulators: the K-norm of the step (Eq. 4), if the caller has one.
-        //      It streams K from HBM, which the Gram tiles (fed from L2) leave idle.  16 lanes per token.
-        if (g.kn_K) {
-            const int d8 = g.kn_d / 8;
-            const int64_t sn = d8, sh = (int64_t)g.kn_N * d8, sb = (int64_t)g.kn_H * sh;
-            const uint4* Kp = static_cast<const uint4*>(g.kn_K);
-            const int sub = e & 15;
-            const long long tokens = (long long)g.B * g.kn_Nv;
-            // a warp serves two consecutive tokens; the loop runs on the warp's first token so that all 32 lanes
-            // stay together for the shuffles
-            for (long long tw = (long long)blockIdx.x * (kResidentEpiThreads / 16) + 2 * (e >> 5); tw < tokens;
-                 tw += (long long)gridDim.x * (kResidentEpiThreads / 16)) {
-                const long long tk = tw + ((e >> 4) & 1);
-                const bool live = tk < tokens;
-                const int b = live ? (int)(tk / g.kn_Nv) : 0, i = live ? (int)(tk - (long long)b * g.kn_Nv) : 0;
-                float part = 0.f;
-                if (live)
-                    part = knorm_token_partial<16, 8>(Kp + b * sb + (int64_t)(g.kn_vis_start + i) * sn, g.kn_H, d8, sh, sub);
-#pragma unroll
-                for (int off = 8; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-                if (live && sub == 0) g.kn_score[(size_t)b * g.kn_Nv + i] = sqrtf(part);
-            }
-        }
         // ---- phase 0: the diagonal tiles give g_ii, hence the per-token factors every other epilogue needs
         uint32_t slot = 0;
         for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
             EpiCall c;
-            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            decode_resident_tile(k, t, c.b, c.ti, c.tj);
             if (c.ti != c.tj) continue;                    // uniform over the CTA
             c.tmem_tile = tmem_base + slot * BN;
             c.wait_bar = bar_tfull + 8 * slot;
@@ -861,16 +1018,18 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             c.rho_from_part = false;
             c.abort_flag = abort_flag;
             stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS>(k, sm, c, ok);
+            if (!stop) resident_publish(g.diag_ready + (size_t)c.b * k.t.TI + c.ti);
         }
-        stop = resident_grid_barrier(g.grid_sync + 1, abort_flag, stop);
-        // Every CTA of this grid is resident now (all have arrived at the barrier), so the kernels that follow may
-        // be scheduled beside it without taking an SM slot one of its CTAs still needs.
-        grid_dependency_launch_dependents();
-        // ---- phase 1: density partials
+        // ---- phase 1: density partials, tile by tile as soon as the factors of its row and column block exist
         slot = 0;
         for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
             EpiCall c;
-            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            decode_resident_tile(k, t, c.b, c.ti, c.tj);
+            if (c.ti != c.tj) {
+                stop = resident_wait_flags(g.diag_ready + (size_t)c.b * k.t.TI + c.ti,
+                                           g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop);
+                if (stop) break;
+            }
             c.tmem_tile = tmem_base + slot * BN;
             c.wait_bar = bar_tfull + 8 * slot;
             c.wait_parity = 0;
@@ -880,12 +1039,15 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS>(k, sm, c, ok);
         }
         stop = resident_grid_barrier(g.grid_sync, abort_flag, stop);
+        // The kernels that follow cannot share an SM with a CTA of this grid (registers, shared memory); from here
+        // on they may at least be set up.
+        grid_dependency_launch_dependents();
         // ---- phase 2: delta and parents from the same accumulators; every tile sums the rho of its own rows and
         //      columns from the partials (fixed order: the same bits everywhere)
         slot = 0;
         for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
             EpiCall c;
-            decode_tile<BN, true, false>(k, t, c.b, c.ti, c.tj);
+            decode_resident_tile(k, t, c.b, c.ti, c.tj);
             c.tmem_tile = tmem_base + slot * BN;
             c.wait_bar = 0;
             c.wait_parity = 0;
@@ -1074,6 +1236,13 @@ bool gram_fits_resident(int B, int n) {
     const long long ti = (n + BM - 1) / BM;
     const long long tiles = (long long)B * ti * (ti + 1) / 2;
     return tiles > 0 && tiles <= (long long)kResidentSlots * num_sms();
+}
+
+bool gram_resident_takes_knorm(int H, int d) {
+    // sixteen or more 16-byte pieces per row (the lane layout of the stand-alone kernel's widest variant), and at
+    // least one chunk of eight tokens must fit the operand buffers
+    if (H <= 0 || d <= 0 || d % 8 || d / 8 < 16) return false;
+    return (long long)H * kKnChunkTokens * d * 2 <= (long long)GemmSmem<BM>::kTileBytes;
 }
 
 int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream) {

@@ -56,12 +56,14 @@ struct GramArgs {
     float* a_out;               // [B, n]
     float* rho_out;             // [B, n] written by the resident sweep (same memory as rho)
     float* rho_user;            // [B, n] optional copy of rho for the caller
-    unsigned int* grid_sync;    // two zeroed counters for the resident sweep's grid-wide barriers
-    // Optional K-norm (Eq. 4) for the resident sweep's epilogue warps to compute while the tensor cores fill the
-    // accumulators: K bf16 [B, kn_H, kn_N, kn_d] dense, span [kn_vis_start, kn_vis_start + kn_Nv), score [B, kn_Nv].
+    unsigned int* grid_sync;    // zeroed counter for the resident sweep's grid-wide barrier
+    unsigned int* diag_ready;   // zeroed flags [B, ceil(n / 128)] of the resident sweep: factors of a row block written
+    // Optional K-norm (Eq. 4) for the resident sweep's load and MMA warps to stream once their own work is issued:
+    // K bf16 [kn_B, kn_H, kn_N, kn_d] dense, span [kn_vis_start, kn_vis_start + kn_Nv), score [kn_B, kn_Nv].
+    // Only shapes gram_resident_takes_knorm accepts.
     const void* kn_K;
     float* kn_score;
-    int kn_H, kn_N, kn_d, kn_vis_start, kn_Nv;
+    int kn_B, kn_H, kn_N, kn_d, kn_vis_start, kn_Nv;
     int* status;                // device status word
 };
 
@@ -72,16 +74,16 @@ __host__ __device__ inline float rho_from_partials(const float* p, const GramTil
     const int ti = i / kGramBM, tj = i / t.BN;
     const int cap = t.R * (tj + 1);
     const int rows = t.TI < cap ? t.TI : cap;
-    // slots [c0, TJ) on the row side, then [TJ, TJ + rows) on the column side: one contiguous walk, loaded eight
+    // slots [c0, TJ) on the row side, then [TJ, TJ + rows) on the column side: one contiguous walk, loaded sixteen
     // at a time (independent loads) and added one by one in slot order
     const int first = ti / t.R, last = t.TJ + rows;
     float s = 0.f;
-    for (int c = first; c < last; c += 8) {
-        float v[8];
+    for (int c = first; c < last; c += 16) {
+        float v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = (c + u < last) ? p[(size_t)(c + u) * t.n_pad] : 0.f;
+        for (int u = 0; u < 16; ++u) v[u] = (c + u < last) ? p[(size_t)(c + u) * t.n_pad] : 0.f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
+        for (int u = 0; u < 16; ++u)
             if (c + u < last) s += v[u];
     }
     return s;
@@ -91,10 +93,14 @@ __host__ __device__ inline float rho_from_partials(const float* p, const GramTil
 // 128 x 128 tiles per SM): density and delta can then share one pass over the Gram tiles (launch_gram_resident).
 bool gram_fits_resident(int B, int n);
 
+// True when the resident sweep can compute the K-norm of keys with H heads of d elements on the side.
+bool gram_resident_takes_knorm(int H, int d);
+
 // One kernel for the norms, Eq. 2 and Eq. 3 on small problems: every CTA keeps the accumulators of its tiles in
-// tensor memory; the grid synchronises (bounded waits) after the diagonal tiles have produced the per-token
-// factors and after the density partials; the delta epilogue sums the partials it needs itself and re-reads the
-// same accumulators.  `tiling` = make_gram_tiling(n, 128).
+// tensor memory; the diagonal tiles publish the per-token factors of their row block behind a flag that the
+// density epilogues of the other tiles wait for, the grid synchronises once (bounded waits) after the density
+// partials; the delta epilogue sums the partials it needs itself and re-reads the same accumulators.
+// `tiling` = make_gram_tiling(n, 128).
 int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream);
 
 // Enqueues one sweep.  `tiling` must come from make_gram_tiling(n, gram_pick_bn(B, n)) for the symmetric modes.

@@ -54,6 +54,8 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
                    void* V_out, int Ncap, int32_t* kept_pos, int32_t* out_len, cudaStream_t stream, bool pdl);
 
 size_t filter_workspace_bytes(int B, int n, int D);
+// Leading bytes of the filter workspace that must be zero when launch_filter starts (status block and flags).
+size_t filter_zeroed_bytes(int B, int n);
 size_t similarity_workspace_bytes(int B, int n, int D);
 int launch_filter(const void* feat, const float* pos, int B, int n, int D, const vitcop_filter_params& p,
                   int n_centers, int32_t* label, int32_t* n_clusters, float* rho, float* delta2, int32_t* parent,

@@ -36,7 +36,9 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
     // Only now may the next kernel's CTAs be scheduled: released earlier they would sit on the SMs waiting for
     // this grid while its own remaining CTAs queue behind them.
     grid_dependency_launch_dependents();
-    if (late_wait) grid_dependency_wait();
+    // One waiting CTA is enough to keep the grid from completing early; the others leave and free their SM slots
+    // for the CTAs of this grid that have not started yet.
+    if (late_wait && blockIdx.x == 0 && blockIdx.y == 0) grid_dependency_wait();
 }
 
 }  // namespace
