@@ -179,7 +179,8 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
 struct KernelArgs {
     GramArgs g;
     GramTiling t;
-    long long total_tiles;
+    long long total_tiles;         // the resident sweep counts its units here
+    int extra_units_per_b;         // resident sweep: units of one sample that do not hold a diagonal tile
 };
 
 template <int BN, bool SYM, bool DIAG = false>
@@ -706,9 +707,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 // the resident kernel: density and delta from ONE pass over the Gram tiles (small problems)
 // ------------------------------------------------------------------------------------------------
-// Every CTA owns at most kResidentSlots tiles of 128 x 128 and keeps all their accumulators in tensor memory
-// (4 x 128 of the 512 columns).  Tiles are numbered with the diagonal ones first, so that these are the first
-// accumulators to complete.  Phases of the epilogue warps:
+// The unit of work is one row block (128 tokens) against two adjacent column blocks: one MMA of N = 256 per
+// k-step, the row operand loaded once for both 128 x 128 tiles (a quarter less operand traffic than tile by tile,
+// and the tensor cores run N = 256 at twice the rate of N = 128).  Row block ti owns the column blocks ti .. TI - 1,
+// paired from the diagonal on; the last unit of a row is half empty when their number is odd (the rows of its
+// missing column block lie outside the tensor and are zero-filled at no cost in traffic).  A CTA owns at most
+// kResidentUnits units and keeps their accumulators in tensor memory (2 x 256 of the 512 columns).  Units that
+// start with a diagonal tile are numbered first, so that these accumulators are the first to complete.
+// Phases of the epilogue warps, which treat a unit as two tiles of 128 x 128:
 //   0. the diagonal tiles yield g_ii -> per-token normalisation factors, published behind one flag per row block
 //   1. density epilogue of every tile (after the flags of its row and column block) -> rho partials;
 //      grid-wide barrier
@@ -721,7 +727,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // operand buffers and -- for the rest of the kernel, which is arithmetic on the accumulators -- the memory system:
 // if the caller has a K-norm (Eq. 4) to compute, these two warps stream K through the operand buffers with bulk
 // copies and reduce it there (resident_knorm).
-constexpr int kResidentSlots = 4;
+constexpr int kResidentUnits = 2;
+constexpr int kResidentBN = 2 * BM;                       // columns of a unit
 constexpr int kResidentEpiThreads = 512;
 
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
@@ -767,25 +774,40 @@ __device__ __forceinline__ bool resident_wait_flags(const unsigned int* fa, cons
     return stop;
 }
 
-// Tile t of the resident sweep: the B * TI diagonal tiles first, then the tiles above the diagonal, sample by
-// sample, column tile by column tile.
-__device__ __forceinline__ void decode_resident_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
+// Unit t of the resident sweep: the B * TI units that start with a diagonal tile first, then the others, sample
+// by sample and row block by row block.
+struct ResidentUnit {
+    int b, ti, tj0;        // sample, row block, first column block
+    int width;             // column blocks inside the tensor: 2, or 1 for the half-empty last unit of a row
+};
+__host__ __device__ inline int resident_extra_units(int TI) {
+    int e = 0;
+    for (int ti = 0; ti < TI; ++ti) e += (TI - ti + 1) / 2 - 1;
+    return e;
+}
+__device__ __forceinline__ ResidentUnit decode_resident_unit(const KernelArgs& k, long long t) {
     const int TI = k.t.TI;
     const long long n_diag = (long long)k.g.B * TI;
+    ResidentUnit u;
     if (t < n_diag) {
-        b = (int)(t / TI);
-        ti = tj = (int)(t - (long long)b * TI);
-        return;
+        u.b = (int)(t / TI);
+        u.ti = (int)(t - (long long)u.b * TI);
+        u.tj0 = u.ti;
+    } else {
+        const long long x = t - n_diag;                    // extra_units_per_b > 0 here
+        u.b = (int)(x / k.extra_units_per_b);
+        int r = (int)(x - (long long)u.b * k.extra_units_per_b);
+        int ti = 0;
+        for (; ti < TI; ++ti) {
+            const int m = (TI - ti + 1) / 2 - 1;           // units of row block ti beyond its first
+            if (r < m) break;
+            r -= m;
+        }
+        u.ti = ti;
+        u.tj0 = ti + 2 * (r + 1);
     }
-    const int above = TI * (TI - 1) / 2;                   // > 0 here: with TI == 1 every tile is diagonal
-    const long long u = t - n_diag;
-    b = (int)(u / above);
-    const int r = (int)(u - (long long)b * above);
-    int q = (int)((sqrtf(8.f * (float)r + 1.f) - 1.f) * 0.5f);
-    while (q > 0 && q * (q + 1) / 2 > r) --q;
-    while ((q + 1) * (q + 2) / 2 <= r) ++q;
-    tj = q + 1;
-    ti = r - q * (q + 1) / 2;
+    u.width = u.tj0 + 1 < TI ? 2 : 1;
+    return u;
 }
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -889,9 +911,9 @@ template <int METRIC, bool SPATIAL>
 __global__ void __launch_bounds__(64 + kResidentEpiThreads, 1)
 gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const KernelArgs k) {
-    constexpr int BN = BM;
+    constexpr int BN = BM;                                 // the epilogue's tiles
     constexpr int NS = 4;
-    using S = GemmSmem<BN>;
+    using S = GemmSmem<kResidentBN>;                       // stages of 128 + 256 operand rows
     const GramArgs& g = k.g;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -900,25 +922,25 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     EpiSmem sm;
     sm.template carve<BN>(gen + S::kTileBytes);
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen + S::kTileBytes + S::kEpiBytes);
-    // barriers: full[kStages], empty[kStages], tmem_full[kResidentSlots], drain, knorm[kKnBuffers]
+    // barriers: full[kStages], empty[kStages], tmem_full[kResidentUnits], drain, knorm[kKnBuffers]
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * S::kStages;
     const uint32_t bar_tfull = bar_empty + 8 * S::kStages;
-    const uint32_t bar_drain = bar_tfull + 8 * kResidentSlots;
+    const uint32_t bar_drain = bar_tfull + 8 * kResidentUnits;
     const uint32_t bar_kn = bar_drain + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + kResidentSlots + 1 + kKnBuffers);
-    static_assert((2 * S::kStages + kResidentSlots + 1 + kKnBuffers) * 8 + 8 <= S::kBarBytes, "barrier block too small");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + kResidentUnits + 1 + kKnBuffers);
+    static_assert((2 * S::kStages + kResidentUnits + 1 + kKnBuffers) * 8 + 8 <= S::kBarBytes, "barrier block too small");
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr uint32_t kTmemCols = kResidentSlots * BN;   // 512: the whole tensor memory of the SM
+    constexpr uint32_t kTmemCols = kResidentUnits * kResidentBN;   // 512: the whole tensor memory of the SM
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::kStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int a = 0; a < kResidentSlots; ++a) mbar_init(bar_tfull + 8 * a, 1);
+        for (int a = 0; a < kResidentUnits; ++a) mbar_init(bar_tfull + 8 * a, 1);
         mbar_init(bar_drain, 1);
         for (int a = 0; a < kKnBuffers; ++a) mbar_init(bar_kn + 8 * a, 1);
         *abort_flag = 0;
@@ -932,7 +954,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const long long total_tiles = k.total_tiles;          // <= kResidentSlots * gridDim.x (checked by the launcher)
+    const long long total_units = k.total_tiles;          // <= kResidentUnits * gridDim.x (checked by the launcher)
     const int KB = g.D / BK;
 
     if (warp == 0) {
@@ -941,16 +963,16 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0, issued_parity = 0;
             bool ok = true;
-            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
-                int b, ti, tj;
-                decode_resident_tile(k, t, b, ti, tj);
-                const int I0 = ti * BM, J0 = tj * BN;
+            for (long long t = blockIdx.x; ok && t < total_units; t += gridDim.x) {
+                const ResidentUnit u = decode_resident_unit(k, t);
+                const int I0 = u.ti * BM, J0 = u.tj0 * BM;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = tiles + stage * S::kStageBytes;
+                    // rows of the box past the sample's last token are zero-filled and still count as received
                     mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
-                    tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
-                    tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, b);
+                    tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, u.b);
+                    tma_load_3d(sa + S::kABytes, &map_b, bar_full + 8 * stage, kb * BK, J0, u.b);
                     issued |= 1u << stage;
                     issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
@@ -962,14 +984,14 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer: tile s of this CTA -> slot s
+        // ------------------------------------------------------------------ MMA issuer: unit s of this CTA -> columns 256 s ..
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, kResidentBN);
             uint32_t stage = 0, phase = 0;
             uint32_t slot = 0;
             bool ok = true;
-            for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x, ++slot) {
-                const uint32_t d_tmem = tmem_base + slot * BN;
+            for (long long t = blockIdx.x; ok && t < total_units; t += gridDim.x, ++slot) {
+                const uint32_t d_tmem = tmem_base + slot * kResidentBN;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -994,49 +1016,50 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (warp < 2) {
         __syncwarp();
         if (g.kn_K) {
-            const long long my_tiles = (total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;   // >= 1
-            resident_knorm(g, gen, tiles, (uint32_t)S::kTileBytes, bar_kn, bar_tfull + 8 * (uint32_t)(my_tiles - 1),
+            const long long my_units = (total_units - blockIdx.x + gridDim.x - 1) / gridDim.x;   // >= 1
+            resident_knorm(g, gen, tiles, (uint32_t)S::kTileBytes, bar_kn, bar_tfull + 8 * (uint32_t)(my_units - 1),
                            abort_flag);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..17)
-        const int e = threadIdx.x - 64;
         bool ok = true;
         bool stop = false;
         grid_dependency_wait();
+        // tile s (0 or 1) of this CTA's unit number `slot`
+        auto tile_call = [&](const ResidentUnit& u, uint32_t slot, int s, bool wait_mma, bool rho_from_part) {
+            EpiCall c;
+            c.b = u.b;
+            c.ti = u.ti;
+            c.tj = u.tj0 + s;
+            c.tmem_tile = tmem_base + slot * kResidentBN + (uint32_t)s * BN;
+            c.wait_bar = wait_mma ? bar_tfull + 8 * slot : 0;
+            c.wait_parity = 0;
+            c.arrive_bar = 0;
+            c.rho_from_part = rho_from_part;
+            c.abort_flag = abort_flag;
+            return c;
+        };
 
         // ---- phase 0: the diagonal tiles give g_ii, hence the per-token factors every other epilogue needs
         uint32_t slot = 0;
-        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
-            EpiCall c;
-            decode_resident_tile(k, t, c.b, c.ti, c.tj);
-            if (c.ti != c.tj) continue;                    // uniform over the CTA
-            c.tmem_tile = tmem_base + slot * BN;
-            c.wait_bar = bar_tfull + 8 * slot;
-            c.wait_parity = 0;
-            c.arrive_bar = 0;
-            c.rho_from_part = false;
-            c.abort_flag = abort_flag;
+        for (long long t = blockIdx.x; t < total_units && !stop; t += gridDim.x, ++slot) {
+            const ResidentUnit u = decode_resident_unit(k, t);
+            if (u.ti != u.tj0) continue;                   // uniform over the CTA
+            const EpiCall c = tile_call(u, slot, 0, true, false);
             stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS>(k, sm, c, ok);
-            if (!stop) resident_publish(g.diag_ready + (size_t)c.b * k.t.TI + c.ti);
+            if (!stop) resident_publish(g.diag_ready + (size_t)u.b * k.t.TI + u.ti);
         }
         // ---- phase 1: density partials, tile by tile as soon as the factors of its row and column block exist
         slot = 0;
-        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
-            EpiCall c;
-            decode_resident_tile(k, t, c.b, c.ti, c.tj);
-            if (c.ti != c.tj) {
-                stop = resident_wait_flags(g.diag_ready + (size_t)c.b * k.t.TI + c.ti,
-                                           g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop);
-                if (stop) break;
+        for (long long t = blockIdx.x; t < total_units && !stop; t += gridDim.x, ++slot) {
+            const ResidentUnit u = decode_resident_unit(k, t);
+            for (int s = 0; s < u.width && !stop; ++s) {
+                const EpiCall c = tile_call(u, slot, s, true, false);
+                if (c.ti != c.tj)
+                    stop = resident_wait_flags(g.diag_ready + (size_t)c.b * k.t.TI + c.ti,
+                                               g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop);
+                if (!stop) stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS>(k, sm, c, ok);
             }
-            c.tmem_tile = tmem_base + slot * BN;
-            c.wait_bar = bar_tfull + 8 * slot;
-            c.wait_parity = 0;
-            c.arrive_bar = 0;
-            c.rho_from_part = false;
-            c.abort_flag = abort_flag;
-            stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS>(k, sm, c, ok);
         }
         stop = resident_grid_barrier(g.grid_sync, abort_flag, stop);
         // The kernels that follow cannot share an SM with a CTA of this grid (registers, shared memory); from here
@@ -1045,16 +1068,12 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // ---- phase 2: delta and parents from the same accumulators; every tile sums the rho of its own rows and
         //      columns from the partials (fixed order: the same bits everywhere)
         slot = 0;
-        for (long long t = blockIdx.x; t < total_tiles && !stop; t += gridDim.x, ++slot) {
-            EpiCall c;
-            decode_resident_tile(k, t, c.b, c.ti, c.tj);
-            c.tmem_tile = tmem_base + slot * BN;
-            c.wait_bar = 0;
-            c.wait_parity = 0;
-            c.arrive_bar = 0;
-            c.rho_from_part = true;
-            c.abort_flag = abort_flag;
-            stop = epi_tile<BN, GRAM_DELTA, METRIC, SPATIAL, NS>(k, sm, c, ok);
+        for (long long t = blockIdx.x; t < total_units && !stop; t += gridDim.x, ++slot) {
+            const ResidentUnit u = decode_resident_unit(k, t);
+            for (int s = 0; s < u.width && !stop; ++s) {
+                const EpiCall c = tile_call(u, slot, s, false, true);
+                stop = epi_tile<BN, GRAM_DELTA, METRIC, SPATIAL, NS>(k, sm, c, ok);
+            }
         }
     }
 
@@ -1167,7 +1186,7 @@ int launch_bn(int mode, const CUtensorMap& ma, const CUtensorMap& mb, const Kern
 
 template <int METRIC, bool SPATIAL>
 int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream) {
-    using S = GemmSmem<BM>;
+    using S = GemmSmem<kResidentBN>;
     static bool attr_done = false;
     auto kern = gram_resident_kernel<METRIC, SPATIAL>;
     if (!attr_done) {
@@ -1175,9 +1194,9 @@ int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const Kern
         if (e != cudaSuccess) return record_cuda(e);
         attr_done = true;
     }
-    const long long ctas = (k.total_tiles + kResidentSlots - 1) / kResidentSlots;
+    const long long ctas = (k.total_tiles + kResidentUnits - 1) / kResidentUnits;
     cudaLaunchConfig_t cfg = {};
-    // as many CTAs as there are SMs (never fewer than the tiles need): the shortest chain of tiles per CTA
+    // as many CTAs as there are SMs (never fewer than the units need): the shortest chain of units per CTA
     cfg.gridDim = dim3((unsigned)(k.total_tiles < num_sms() ? k.total_tiles : (ctas > num_sms() ? ctas : num_sms())));
     cfg.blockDim = dim3(64 + kResidentEpiThreads);
     cfg.dynamicSmemBytes = S::kTotal;
@@ -1233,16 +1252,16 @@ bool gram_fits_resident(int B, int n) {
                        cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 0;
     }
     if (!cooperative) return false;
-    const long long ti = (n + BM - 1) / BM;
-    const long long tiles = (long long)B * ti * (ti + 1) / 2;
-    return tiles > 0 && tiles <= (long long)kResidentSlots * num_sms();
+    const int ti = (n + BM - 1) / BM;
+    const long long units = (long long)B * (ti + resident_extra_units(ti));
+    return units > 0 && units <= (long long)kResidentUnits * num_sms();
 }
 
 bool gram_resident_takes_knorm(int H, int d) {
     // sixteen or more 16-byte pieces per row (the lane layout of the stand-alone kernel's widest variant), and at
     // least one chunk of eight tokens must fit the operand buffers
     if (H <= 0 || d <= 0 || d % 8 || d / 8 < 16) return false;
-    return (long long)H * kKnChunkTokens * d * 2 <= (long long)GemmSmem<BM>::kTileBytes;
+    return (long long)H * kKnChunkTokens * d * 2 <= (long long)GemmSmem<kResidentBN>::kTileBytes;
 }
 
 int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream) {
@@ -1251,11 +1270,13 @@ int launch_gram_resident(const void* feat, const GramArgs& args, const GramTilin
     k.t = tiling;
     k.g.row0 = 0;
     k.g.row_end = args.n;
-    k.total_tiles = (long long)args.B * k.t.tiles_per_b;
+    k.extra_units_per_b = resident_extra_units(k.t.TI);
+    k.total_tiles = (long long)args.B * (k.t.TI + k.extra_units_per_b);
     if (k.total_tiles <= 0) return VITCOP_OK;
-    if (tiling.BN != BM || k.total_tiles > (long long)kResidentSlots * num_sms()) return VITCOP_ERR_INVALID_ARG;
+    if (tiling.BN != BM || k.total_tiles > (long long)kResidentUnits * num_sms()) return VITCOP_ERR_INVALID_ARG;
     CUtensorMap ma, mb;
-    if (!make_feat_map(&ma, feat, args.B, args.n, args.D, BM) || !make_feat_map(&mb, feat, args.B, args.n, args.D, BM))
+    if (!make_feat_map(&ma, feat, args.B, args.n, args.D, BM) ||
+        !make_feat_map(&mb, feat, args.B, args.n, args.D, kResidentBN))
         return VITCOP_ERR_CUDA;
     const bool euclid = args.metric == 1;
     const bool spatial = args.tau2 >= 0.f && args.pos != nullptr;
