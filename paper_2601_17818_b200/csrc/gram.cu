@@ -135,6 +135,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
     for (int u = 0; u < 32; ++u) v[u] = __uint_as_float(r[u]);
 }
+// 8 consecutive fp32 columns of this thread's TMEM lane: the load is asynchronous, the registers hold the data only
+// after tmem_ld8_wait on the same registers (the wait names them, so no use of theirs can be moved in front of it).
+__device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld8_wait(uint32_t (&r)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+                 :
+                 : "memory");
+}
 template <int THREADS>
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 // Barrier over the epilogue threads that also ORs a predicate: every thread gets the same answer.
@@ -217,6 +232,18 @@ __device__ __forceinline__ void butterfly_stage(float* v, bool up) {
         v[k] = MIN ? fminf(keep, recv) : keep + recv;
     }
 }
+// Eight columns held by every lane (one row each): afterwards every lane holds the sum over the 32 lanes of column
+// lane & 7, added in a fixed order.
+__device__ __forceinline__ float warp_column_sums8(float (&v)[8], int lane) {
+    butterfly_stage<4, false>(v, (lane & 4) != 0);
+    butterfly_stage<2, false>(v, (lane & 2) != 0);
+    butterfly_stage<1, false>(v, (lane & 1) != 0);
+    float s = v[0];
+    s += __shfl_xor_sync(0xffffffffu, s, 8);
+    s += __shfl_xor_sync(0xffffffffu, s, 16);
+    return s;
+}
+__device__ __forceinline__ float column_sums(float (&v)[8], int lane) { return warp_column_sums8(v, lane); }
 template <bool MIN>
 __device__ __forceinline__ float warp_transpose_reduce(float (&v)[32], int lane) {
     butterfly_stage<16, MIN>(v, (lane & 16) != 0);
@@ -226,6 +253,8 @@ __device__ __forceinline__ float warp_transpose_reduce(float (&v)[32], int lane)
     butterfly_stage<1, MIN>(v, (lane & 1) != 0);
     return v[0];
 }
+
+__device__ __forceinline__ float column_sums(float (&v)[32], int lane) { return warp_transpose_reduce<false>(v, lane); }
 
 // ------------------------------------------------------------------------------------------------
 // shared memory
@@ -282,13 +311,17 @@ struct EpiCall {
 };
 
 // Returns true when the CTA must give up (a bounded wait expired somewhere).
-template <int BN, int MODE, int METRIC, bool SPATIAL, int NS>
+// GW: columns a warp takes from the accumulator at a time.  32 unrolls the whole arithmetic of a 32-column chunk
+// (fewest instructions; right where the code is reused tile after tile), 8 keeps it in a short rolled loop (right
+// where every tile is visited once and the instruction cache would otherwise miss all the way).
+template <int BN, int MODE, int METRIC, bool SPATIAL, int NS, int GW = 32>
 __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm, const EpiCall& call, bool& ok) {
+    static_assert(GW == 8 || GW == 32, "group width");
     constexpr bool SYM = MODE == GRAM_RHO || MODE == GRAM_DELTA;
     constexpr bool DIAG = MODE == GRAM_DIAG;
     constexpr int kEpiThreads = NS * 128;
     constexpr int kSliceCols = BN / NS;
-    constexpr int kChunks = kSliceCols / 32;           // 32-column chunks per warp
+    constexpr int kGroups = kSliceCols / GW;           // column groups per warp, taken one by one in a rolled loop
     const GramArgs& g = k.g;
     float *colw = sm.colw, *cola = sm.cola, *colrho = sm.colrho, *colx = sm.colx, *coly = sm.coly;
     float *colred = sm.colred, *rowred = sm.rowred;
@@ -376,24 +409,36 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
     if (ok) {
         tc_fence_after();
         const uint32_t taddr = call.tmem_tile + ((uint32_t)(quarter * 32) << 16) + slice * kSliceCols;
+        uint32_t ld_cur[8], ld_nxt[8];
+        if constexpr (GW == 8) {
+            tmem_ld8_issue(taddr, ld_cur);
+            tmem_ld8_wait(ld_cur);
+        }
 #pragma unroll 1
-        for (int c = 0; c < kChunks; ++c) {
-            float v[32];
-            tmem_ld32(taddr + c * 32, v);
-            if (c == kChunks - 1) {
+        for (int c = 0; c < kGroups; ++c) {
+            float v[GW];
+            if constexpr (GW == 8) {
+                // the next group's accumulators travel while this one is worked on
+                if (c + 1 < kGroups) tmem_ld8_issue(taddr + (c + 1) * 8, ld_nxt);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __uint_as_float(ld_cur[u]);
+            } else {
+                tmem_ld32(taddr + c * 32, v);
+            }
+            if (c == kGroups - 1) {
                 // this thread has read all it needs from the accumulator
                 tc_fence_before();
                 if (call.arrive_bar) mbar_arrive(call.arrive_bar);
             }
-            const int cl0 = slice * kSliceCols + c * 32;       // tile-local first column of the chunk
+            const int cl0 = slice * kSliceCols + c * GW;       // tile-local first column of the group
             const float4* cw4 = reinterpret_cast<const float4*>(colw + cl0);
             const float4* ca4 = reinterpret_cast<const float4*>(cola + cl0);
             if (MODE == GRAM_DIAG) {
-                // g_ii sits in column rl of row rl: the chunk that starts at this warp's first row
-                if (cl0 == quarter * 32 && row_valid) {
+                // g_ii sits in column rl of row rl
+                if (cl0 == (rl & ~(GW - 1)) && row_valid) {
                     float gii = 0.f;
 #pragma unroll
-                    for (int u = 0; u < 32; ++u) gii = (u == lane) ? v[u] : gii;
+                    for (int u = 0; u < GW; ++u) gii = (u == (lane & (GW - 1))) ? v[u] : gii;
                     // The squared norm comes from the same tensor-core arithmetic as every g_ij, so the
                     // rounding of the accumulation cancels in s_ij = g_ij / sqrt(g_ii g_jj) where it
                     // matters: near-duplicates (s -> 1, d^2 = 2 - 2 s -> 0); exact duplicates give s = 1.
@@ -405,7 +450,7 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                 if (row_valid) {
                     float* o = g.sim_out + ((size_t)b * rows_out + (i - g.row0)) * g.n;
 #pragma unroll
-                    for (int u = 0; u < 32; ++u) {
+                    for (int u = 0; u < GW; ++u) {
                         const int j = J0 + cl0 + u;
                         if (j < g.n) o[j] = METRIC == 0 ? (v[u] * w_i) * colw[cl0 + u] : v[u];
                     }
@@ -413,7 +458,7 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
             } else if (MODE == GRAM_RHO) {
                 // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
 #pragma unroll
-                for (int q4 = 0; q4 < 8; ++q4) {
+                for (int q4 = 0; q4 < GW / 4; ++q4) {
                     const float4 cw = cw4[q4];
                     float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (METRIC == 1) ca = ca4[q4];
@@ -430,22 +475,22 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                 }
                 if (!full) {
 #pragma unroll
-                    for (int u = 0; u < 32; ++u) {
+                    for (int u = 0; u < GW; ++u) {
                         const int j = J0 + cl0 + u;
                         v[u] = (j > i && j < g.n && row_valid) ? v[u] : 0.f;
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < 32; ++u) racc += v[u];
-                const float cs = warp_transpose_reduce<false>(v, lane);
-                colred[quarter * BN + cl0 + lane] = cs;
+                for (int u = 0; u < GW; ++u) racc += v[u];
+                const float cs = column_sums(v, lane);
+                if (lane < GW) colred[quarter * BN + cl0 + lane] = cs;
             } else {  // GRAM_DELTA, Eq. 3
                 const float4* cr4 = reinterpret_cast<const float4*>(colrho + cl0);
                 const float4* cx4 = reinterpret_cast<const float4*>(colx + cl0);
                 const float4* cy4 = reinterpret_cast<const float4*>(coly + cl0);
-                uint32_t kc[32];                   // column-side keys: d^2 >= 0 orders like its bit pattern
+                uint32_t kc[GW];                   // column-side keys: d^2 >= 0 orders like its bit pattern
 #pragma unroll
-                for (int q4 = 0; q4 < 8; ++q4) {
+                for (int q4 = 0; q4 < GW / 4; ++q4) {
                     const float4 cw = cw4[q4];
                     const float4 cr = cr4[q4];
                     float4 ca = make_float4(0.f, 0.f, 0.f, 0.f), cx = ca, cy = ca;
@@ -482,14 +527,23 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                 // column side: minimum over this warp's 32 rows and the lowest row that attains it
                 uint32_t my_min = 0x7f800000u, my_rows = 0;
 #pragma unroll
-                for (int u = 0; u < 32; ++u) {
+                for (int u = 0; u < GW; ++u) {
                     const uint32_t m = __reduce_min_sync(0xffffffffu, kc[u]);
                     const uint32_t rows = __ballot_sync(0xffffffffu, kc[u] == m);
                     if (lane == u) { my_min = m; my_rows = rows; }
                 }
-                colred[quarter * BN + cl0 + lane] = __uint_as_float(my_min);
-                colidx[quarter * BN + cl0 + lane] =
-                    my_min < 0x7f800000u ? I0 + quarter * 32 + (__ffs(my_rows) - 1) : -1;
+                if (lane < GW) {
+                    colred[quarter * BN + cl0 + lane] = __uint_as_float(my_min);
+                    colidx[quarter * BN + cl0 + lane] =
+                        my_min < 0x7f800000u ? I0 + quarter * 32 + (__ffs(my_rows) - 1) : -1;
+                }
+            }
+            if constexpr (GW == 8) {
+                if (c + 1 < kGroups) {
+                    tmem_ld8_wait(ld_nxt);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) ld_cur[u] = ld_nxt[u];
+                }
             }
         }
     }
@@ -1046,7 +1100,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const ResidentUnit u = decode_resident_unit(k, t);
             if (u.ti != u.tj0) continue;                   // uniform over the CTA
             const EpiCall c = tile_call(u, slot, 0, true, false);
-            stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS>(k, sm, c, ok);
+            stop = epi_tile<BN, GRAM_DIAG, METRIC, false, NS, 8>(k, sm, c, ok);
             if (!stop) resident_publish(g.diag_ready + (size_t)u.b * k.t.TI + u.ti);
         }
         // ---- phase 1: density partials, tile by tile as soon as the factors of its row and column block exist
@@ -1058,7 +1112,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 if (c.ti != c.tj)
                     stop = resident_wait_flags(g.diag_ready + (size_t)c.b * k.t.TI + c.ti,
                                                g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop);
-                if (!stop) stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS>(k, sm, c, ok);
+                if (!stop) stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS, 8>(k, sm, c, ok);
             }
         }
         stop = resident_grid_barrier(g.grid_sync, abort_flag, stop);
@@ -1072,7 +1126,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const ResidentUnit u = decode_resident_unit(k, t);
             for (int s = 0; s < u.width && !stop; ++s) {
                 const EpiCall c = tile_call(u, slot, s, false, true);
-                stop = epi_tile<BN, GRAM_DELTA, METRIC, SPATIAL, NS>(k, sm, c, ok);
+                stop = epi_tile<BN, GRAM_DELTA, METRIC, SPATIAL, NS, 8>(k, sm, c, ok);
             }
         }
     }
