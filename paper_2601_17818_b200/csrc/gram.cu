@@ -792,26 +792,29 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
 }
 
 // Barrier over all CTAs of the grid, called by the epilogue threads.  Returns true when the grid must give up.
+// One thread speaks for the CTA: the CTA barrier orders every epilogue thread's writes before that thread's fence
+// (and its fence before their later reads), so the other threads need none of their own.
 __device__ __forceinline__ bool resident_grid_barrier(unsigned int* counter, volatile int* abort_flag, bool aborted) {
-    __threadfence();                                       // this thread's global writes are visible device-wide
     epi_bar_sync<kResidentEpiThreads>();
     if (threadIdx.x == 64 && !aborted) {
+        __threadfence();
         atomicAdd(counter, 1u);
         const unsigned long long t0 = global_ns();
         while (ld_acquire_u32(counter) < gridDim.x) {
             if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
         }
+        __threadfence();
     }
-    const bool stop = epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
-    __threadfence();
-    return stop;
+    return epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
 }
 
 // Raises a flag once every epilogue thread's global writes are visible device-wide.
 __device__ __forceinline__ void resident_publish(unsigned int* flag) {
-    __threadfence();
     epi_bar_sync<kResidentEpiThreads>();
-    if (threadIdx.x == 64) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
+    if (threadIdx.x == 64) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
+    }
 }
 
 // Waits (bounded) until both flags are up.  Returns true when the grid must give up.
@@ -822,10 +825,9 @@ __device__ __forceinline__ bool resident_wait_flags(const unsigned int* fa, cons
         while (ld_acquire_u32(fa) == 0u || ld_acquire_u32(fb) == 0u) {
             if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
         }
+        __threadfence();
     }
-    const bool stop = epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
-    __threadfence();
-    return stop;
+    return epi_bar_or<kResidentEpiThreads>(aborted || *abort_flag != 0);
 }
 
 // Unit t of the resident sweep: the B * TI units that start with a diagonal tile first, then the others, sample
