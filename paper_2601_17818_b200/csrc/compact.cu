@@ -2,8 +2,8 @@
 //
 // One CTA per (output row, sample).  The source position of the row comes from the ascending
 // keep list; the CTA then moves the hidden row and the row of every K and V head with 128-bit
-// loads that are all issued before the first store, so that each thread keeps several
-// independent 16-byte requests in flight.  Dropped rows are never read.
+// loads, up to eight of them issued before the first store and taken from all three tensors alike, so that
+// each thread keeps several independent 16-byte requests in flight.  Dropped rows are never read.
 #include "internal.cuh"
 
 namespace vitcop {
@@ -24,40 +24,58 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                  : "memory");
 }
 
-// Copies `total` 16-byte pieces that sit in segments of `seg_len` pieces each (segment s starts at
-// src + s * src_stride / dst + s * dst_stride): one hidden row is a single segment, the K (or V) rows of one
-// token are H segments of d/8 pieces.  Four loads are issued before the first store.
-__device__ __forceinline__ void copy_segments(const uint4* __restrict__ src, uint4* __restrict__ dst, int seg_len,
-                                              int total, int64_t src_stride, int64_t dst_stride, int shift) {
-    for (int q0 = threadIdx.x; q0 < total; q0 += 4 * kCompactThreads) {
-        uint4 v[4];
-        uint4* d[4];
+// Moves one token: its hidden row (dh8 pieces of 16 bytes, one run) and its row in each of the H heads of K and of
+// V (d8 pieces per head, heads head_in / head_out pieces apart).  The pieces of all three tensors form one index
+// space, so that a thread has up to eight loads from any of them in flight before its first store: the row costs
+// one round trip to memory, not one per tensor.  Null tensors are skipped.
+__device__ __forceinline__ void copy_token(const uint4* __restrict__ hid_src, uint4* __restrict__ hid_dst, int dh8,
+                                           const uint4* __restrict__ k_src, uint4* __restrict__ k_dst,
+                                           const uint4* __restrict__ v_src, uint4* __restrict__ v_dst, int H, int d8,
+                                           int d8_shift, int64_t head_in, int64_t head_out) {
+    const int n_hid = hid_src ? dh8 : 0;
+    const int n_kv = H * d8;
+    const int n_k = k_src ? n_kv : 0;
+    const int total = n_hid + n_k + (v_src ? n_kv : 0);
+    constexpr int kInFlight = 8;
+    for (int q0 = threadIdx.x; q0 < total; q0 += kInFlight * kCompactThreads) {
+        uint4 v[kInFlight];
+        uint4* d[kInFlight];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int q = q0 + u * kCompactThreads;
+        for (int u = 0; u < kInFlight; ++u) {
+            int q = q0 + u * kCompactThreads;
             d[u] = nullptr;
             if (q < total) {
-                const int sgm = shift >= 0 ? q >> shift : q / seg_len;
-                const int e = q - sgm * seg_len;
-                v[u] = ld_stream(src + sgm * src_stride + e);
-                d[u] = dst + sgm * dst_stride + e;
+                if (q < n_hid) {
+                    v[u] = ld_stream(hid_src + q);
+                    d[u] = hid_dst + q;
+                } else {
+                    q -= n_hid;
+                    const bool is_k = q < n_k;
+                    if (!is_k) q -= n_k;
+                    const int head = d8_shift >= 0 ? q >> d8_shift : q / d8;
+                    const int e = q - head * d8;
+                    v[u] = ld_stream((is_k ? k_src : v_src) + head * head_in + e);
+                    d[u] = (is_k ? k_dst : v_dst) + head * head_out + e;
+                }
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < kInFlight; ++u)
             if (d[u]) st_stream(d[u], v[u]);
     }
 }
 
-__global__ void __launch_bounds__(kCompactThreads)
-compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, const uint4* __restrict__ V, int H, int N,
+__global__ void __launch_bounds__(kCompactThreads, 4)
+compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, const uint4* __restrict__ V, int B, int H, int N,
                int d8, int dh8, int d8_shift, const int32_t* __restrict__ seq_len, int vis_start,
                const int32_t* __restrict__ vis_len, int vis_len_uniform, const int32_t* __restrict__ keep_idx,
                int keep_stride, const int32_t* __restrict__ n_keep, uint4* __restrict__ hidden_out,
                uint4* __restrict__ K_out, uint4* __restrict__ V_out, int Ncap, int32_t* __restrict__ kept_pos,
                int32_t* __restrict__ out_len) {
-    const int b = blockIdx.y;
-    const int r = blockIdx.x;
+    // CTAs are handed out sample by sample within a row: all the rows in front of the visual span, which need not
+    // wait for the selection, start before the rows that do
+    const int r = (int)(blockIdx.x / (unsigned)B);
+    const int b = (int)(blockIdx.x - (unsigned)r * (unsigned)B);
     const int L = seq_len ? min(seq_len[b], N) : N;
     const int64_t head_in = (int64_t)N * d8, head_out = (int64_t)Ncap * d8;
     // A row in front of the visual span keeps its place whatever the selection turns out to be: it is copied
@@ -65,15 +83,10 @@ compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, co
     // tensors copied here are inputs of the whole call, complete before its first kernel started.)
     const bool prefix_row = r < min(vis_start, L) && r < Ncap;
     if (prefix_row) {
-        if (hidden)
-            copy_segments(hidden + ((int64_t)b * N + r) * dh8, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8, dh8, 0,
-                          0, 31);
-        if (K)
-            copy_segments(K + ((int64_t)b * H * N + r) * d8, K_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
-                          head_in, head_out, d8_shift);
-        if (V)
-            copy_segments(V + ((int64_t)b * H * N + r) * d8, V_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
-                          head_in, head_out, d8_shift);
+        copy_token(hidden ? hidden + ((int64_t)b * N + r) * dh8 : nullptr, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8,
+                   K ? K + ((int64_t)b * H * N + r) * d8 : nullptr, K_out + ((int64_t)b * H * Ncap + r) * d8,
+                   V ? V + ((int64_t)b * H * N + r) * d8 : nullptr, V_out + ((int64_t)b * H * Ncap + r) * d8, H, d8,
+                   d8_shift, head_in, head_out);
         if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = r;
         if (r != 0) return;                                // row 0 still reports the sample's new length
     }
@@ -97,15 +110,10 @@ compact_kernel(const uint4* __restrict__ hidden, const uint4* __restrict__ K, co
     } else src_row = r - nk + nv;
     if (kept_pos && threadIdx.x == 0) kept_pos[(int64_t)b * Ncap + r] = src_row;
 
-    if (hidden)
-        copy_segments(hidden + ((int64_t)b * N + src_row) * dh8, hidden_out + ((int64_t)b * Ncap + r) * dh8, dh8, dh8, 0,
-                      0, 31);
-    if (K)
-        copy_segments(K + ((int64_t)b * H * N + src_row) * d8, K_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
-                      head_in, head_out, d8_shift);
-    if (V)
-        copy_segments(V + ((int64_t)b * H * N + src_row) * d8, V_out + ((int64_t)b * H * Ncap + r) * d8, d8, H * d8,
-                      head_in, head_out, d8_shift);
+    copy_token(hidden ? hidden + ((int64_t)b * N + src_row) * dh8 : nullptr, hidden_out + ((int64_t)b * Ncap + r) * dh8,
+               dh8, K ? K + ((int64_t)b * H * N + src_row) * d8 : nullptr, K_out + ((int64_t)b * H * Ncap + r) * d8,
+               V ? V + ((int64_t)b * H * N + src_row) * d8 : nullptr, V_out + ((int64_t)b * H * Ncap + r) * d8, H, d8,
+               d8_shift, head_in, head_out);
 }
 
 }  // namespace
@@ -122,7 +130,7 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
     cudaLaunchConfig_t cfg = {};
     // rows past min(N, Ncap) cannot exist; one extra CTA row keeps out_len written when Ncap == 0
     const int rows = Ncap > 0 ? Ncap : 1;
-    cfg.gridDim = dim3(rows, B);
+    cfg.gridDim = dim3((unsigned)((long long)B * rows));
     cfg.blockDim = dim3(kCompactThreads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -133,7 +141,7 @@ int launch_compact(const void* hidden, const void* K, const void* V, int B, int 
     KernelTimeScope timed("compact_kernel", stream);
     return record_cuda(cudaLaunchKernelEx(
         &cfg, compact_kernel, static_cast<const uint4*>(hidden), static_cast<const uint4*>(K),
-        static_cast<const uint4*>(V), H, N, d / 8, Dh / 8, d8_shift, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
+        static_cast<const uint4*>(V), B, H, N, d / 8, Dh / 8, d8_shift, seq_len, vis_start, vis_len, vis_len_uniform, keep_idx,
         keep_stride, n_keep, static_cast<uint4*>(hidden_out), static_cast<uint4*>(K_out), static_cast<uint4*>(V_out),
         Ncap, kept_pos, out_len));
 }
