@@ -260,7 +260,10 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
     for name, (launches, ms) in per_kernel.items():
         us = ms * 1e3 / max(launches, 1)
         e = {"launches": launches, "us_per_launch": us}
-        if name in algo and us > 0:
+        if name == "knorm_kernel" and "gram_resident_kernel" in per_kernel:
+            # the step's K-norm is split: some samples inside gram_resident_kernel, the others in this kernel
+            e["note"] = "covers part of the samples only; the rest is computed inside gram_resident_kernel"
+        elif name in algo and us > 0:
             bound, units = algo[name]
             if bound == "hbm":
                 ach, peak, unit = units / (us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"

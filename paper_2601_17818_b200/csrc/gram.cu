@@ -436,9 +436,15 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
             if (MODE == GRAM_DIAG) {
                 // g_ii sits in column rl of row rl
                 if (cl0 == (rl & ~(GW - 1)) && row_valid) {
+                    // (selected with explicit selp: left to itself the compiler indexes the array in local
+                    // memory, a cold round trip on the path every other tile waits for)
                     float gii = 0.f;
+                    const int mine = lane & (GW - 1);
 #pragma unroll
-                    for (int u = 0; u < GW; ++u) gii = (u == (lane & (GW - 1))) ? v[u] : gii;
+                    for (int u = 0; u < GW; ++u)
+                        asm("{\n\t.reg .pred p;\n\tsetp.eq.s32 p, %2, %3;\n\tselp.f32 %0, %1, %0, p;\n\t}"
+                            : "+f"(gii)
+                            : "f"(v[u]), "r"(mine), "r"(u));
                     // The squared norm comes from the same tensor-core arithmetic as every g_ij, so the
                     // rounding of the accumulation cancels in s_ij = g_ij / sqrt(g_ii g_jj) where it
                     // matters: near-duplicates (s -> 1, d^2 = 2 - 2 s -> 0); exact duplicates give s = 1.

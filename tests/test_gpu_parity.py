@@ -364,6 +364,22 @@ def test_filter_small(name, metric, tau):
     print("filter report", name, metric, tau, rep)
 
 
+# Shapes of the one-kernel ("resident") sweep: one or two row blocks, a ragged last block, an odd and an even number
+# of column blocks per row, and enough samples that every SM holds two units of work.
+@pytest.mark.parametrize("B,n,metric,check", [(1, 129, 0, 1), (5, 300, 1, 2), (40, 257, 0, 3), (2, 1000, 0, 2),
+                                              (3, 640, 0, 2)])
+def test_filter_resident_shapes(B, n, metric, check):
+    w = W.workload("tiny")
+    f = W.make_features(w, n=n, B=B)
+    p = np.tile(W.make_positions(w, n)[:1], (B, 1, 1))
+    d_c = w.d_c if metric == 0 else 8.0 * 4
+    nc = max(1, n // 20)
+    g = gpu_filter(f, p, metric, d_c, w.tau, nc)
+    assert g.status == vb.OK and np.all(g.n_clusters == nc)
+    for b in sorted({0, B // 2, B - 1})[:check]:
+        check_vic_sample(f[b], p[b], metric, d_c, w.tau, nc, g.rho[b], g.delta2[b], g.parent[b], g.label[b])
+
+
 def test_filter_edge_cases():
     w = W.workload("tiny")
     # identical tokens: one cluster led by token 0
