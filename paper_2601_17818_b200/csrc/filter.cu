@@ -73,6 +73,9 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t s_digit, s_krem, s_whole;
+    __shared__ unsigned long long orph_best[kFinThreads];
+    __shared__ int orph_list[kFinThreads];
+    __shared__ int orph_cnt;
 
     grid_dependency_launch_dependents();
     grid_dependency_wait();
@@ -209,13 +212,25 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
     }
     __syncthreads();
     if (nc > 0) {
-        for (int o = warp; o < n; o += kFinThreads / 32) {
-            if (isc[o] || nxt[o] != o) continue;                   // only surplus orphans (warp-uniform)
-            const uint16_t* fo = feat + (size_t)o * D;
-            float bestd = __int_as_float(0x7f800000);
-            int bestc = centres[0];
-            for (int q = 0; q < nc; ++q) {
-                const int c = centres[q];
+        // Surplus orphans (roots that are not centres) are rare but each needs its distance to every centre: they
+        // are listed, kFinThreads tokens at a time, and the (orphan, centre) pairs are spread over all warps; the
+        // nearest centre wins through a packed minimum (distance bits, then the lower centre rank).
+        for (int base = 0; base < n; base += kFinThreads) {
+            __syncthreads();                                        // the previous round's list has been consumed
+            if (tid == 0) orph_cnt = 0;
+            __syncthreads();
+            const int o = base + tid;
+            if (o < n && !isc[o] && nxt[o] == o) {
+                const int at = atomicAdd(&orph_cnt, 1);
+                orph_list[at] = o;
+                orph_best[at] = ~0ull;
+            }
+            __syncthreads();
+            const int pairs = orph_cnt * nc;
+            for (int pr = warp; pr < pairs; pr += kFinThreads / 32) {
+                const int e = pr / nc, q = pr - e * nc;
+                const int oo = orph_list[e], c = centres[q];
+                const uint16_t* fo = feat + (size_t)oo * D;
                 const uint16_t* fc = feat + (size_t)c * D;
                 float dot = 0.f;
                 for (int k = lane * 2; k < D; k += 64) {
@@ -226,10 +241,13 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
                 }
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-                const float d2 = fmaxf(0.f, fmaf(-2.f, (dot * w[o]) * w[c], a[o] + a[c]));
-                if (d2 < bestd) { bestd = d2; bestc = c; }
+                const float d2 = fmaxf(0.f, fmaf(-2.f, (dot * w[oo]) * w[c], a[oo] + a[c]));
+                if (lane == 0)
+                    atomicMin(&orph_best[e], ((unsigned long long)__float_as_uint(d2) << 32) | (unsigned long long)q);
             }
-            if (lane == 0) nxt[o] = -1 - bestc;                      // remember the adopted centre at the root
+            __syncthreads();
+            if (tid < orph_cnt)                                     // remember the adopted centre at the root
+                nxt[orph_list[tid]] = -1 - centres[(int)(orph_best[tid] & 0xFFFFFFFFull)];
         }
     }
     __syncthreads();
@@ -352,7 +370,7 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
 
     const int nc = n_centers < n ? n_centers : n;
     const size_t smem = (size_t)n * 8 + (((size_t)n + 15) & ~(size_t)15) + (size_t)(nc > 0 ? nc : 1) * 4 + 16;
-    if (smem > 48 * 1024) {
+    if (smem > 32 * 1024) {                                // (the kernel's static arrays take part of the default 48 KB)
         cudaError_t e = cudaFuncSetAttribute(vic_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda(e);
     }
