@@ -38,9 +38,9 @@ UNIT = "tokens/s"
 # (bytes per launch on the bench workload, sha1 of the kernel's source file when the counters were taken).
 # A kernel whose source changed since reports traffic null.
 NCU_TRAFFIC = {
-    "gram_resident_kernel": (94523904 + 3087360, "42ee52f3e8bd"),
-    "knorm_kernel": (75522560 + 1326848, "6accb3df2988"),
-    "compact_kernel": (33764864 + 976896, "619ac324b74f"),
+    "gram_resident_kernel": (42615040 + 256, "809e93381ca4"),       # features + the keys of its share of the K-norm
+    "knorm_kernel": (51929856 + 19712, "8b9e2bc93897"),             # the samples the resident sweep leaves (11 of 16)
+    "compact_kernel": (33756928 + 882432, "9a7b3fc1ee4a"),
 }
 
 
@@ -263,6 +263,8 @@ def kernel_rooflines(w, nk_total, per_kernel, peaks):
         if name == "knorm_kernel" and "gram_resident_kernel" in per_kernel:
             # the step's K-norm is split: some samples inside gram_resident_kernel, the others in this kernel
             e["note"] = "covers part of the samples only; the rest is computed inside gram_resident_kernel"
+            if w.name == "c1" and NCU_TRAFFIC[name][1] == source_sha(src[name]):
+                e["traffic"] = NCU_TRAFFIC[name][0]
         elif name in algo and us > 0:
             bound, units = algo[name]
             if bound == "hbm":
