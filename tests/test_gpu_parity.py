@@ -1,4 +1,6 @@
 """GPU-vs-oracle parity of the whole pruning chain, through the C ABI (``-m gpu``)."""
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -424,12 +426,17 @@ def test_filter_then_quota_step_end_to_end():
 
 
 # ======================================================================================= Stage II in one call
-@pytest.mark.parametrize("name", ["tiny", "c0", "c1", "c2"])
+# "tiny-wide": six samples of 203 tokens (ragged last chunk of eight), 3 heads of 256 -- a shape whose K-norm the
+# one-kernel sweep takes in part (two 16-byte piece rounds per row), with the rest in the stand-alone kernel.
+@pytest.mark.parametrize("name", ["tiny", "tiny-wide", "c0", "c1", "c2"])
 def test_collaborative_step_equals_filter_then_prune_step(name):
     """vitcop_collaborative_step may reorder its kernels (the K-norm runs beside the clustering) but must return
     exactly what vitcop_redundancy_filter followed by vitcop_prune_step returns; that pair is checked against the
     oracle by the tests above."""
-    w = W.workload(name)
+    if name == "tiny-wide":
+        w = dataclasses.replace(W.workload("tiny"), B=6, Nv=203, H=3, d=256)
+    else:
+        w = W.workload(name)
     B, n = w.B, w.Nv
     feat, pos = vb.bf16_tensor(W.make_features(w)), torch.from_numpy(W.make_positions(w).copy()).to(DEV)
     K_b, V_b = W.make_kv(w, 0, n)
