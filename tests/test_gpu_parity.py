@@ -128,6 +128,23 @@ def test_select_quota_exact(kind, skew):
             assert status == vb.ERR_BUDGET and np.all(nk == 0)
 
 
+@pytest.mark.parametrize("n,ncl,skew", [(64, 5, 0.0), (600, 20, 0.7), (5000, 40, 0.0), (5000, 40, 0.7)])
+def test_select_quota_special_values(n, ncl, skew):
+    """NaN (ranked after everything), infinities, signed zeros and many exact ties, through each search strategy."""
+    rng = np.random.default_rng(n + ncl)
+    score = rng.integers(0, 12, size=(2, n)).astype(np.float32)          # heavy ties
+    special = np.array([np.nan, np.inf, -np.inf, 0.0, -0.0], dtype=np.float32)
+    hit = rng.random((2, n)) < 0.1
+    score[hit] = special[rng.integers(0, len(special), size=int(hit.sum()))]
+    label = W.make_labels(n + 3, 2, n, ncl, skew=skew)
+    for budget in (ncl + 1, (n + ncl) // 3, n):
+        keeps, nk, _, status = gpu_select(score, budget, label=label)
+        assert status == vb.OK
+        for b in range(2):
+            want, nc, _ = oracle.select_quota(score[b].astype(np.float64), label[b], budget)
+            assert np.array_equal(keeps[b], want), (n, ncl, skew, budget)
+
+
 # ======================================================================================= compaction
 def _rand_bits(rng, shape):
     return rng.integers(0, 65536, size=shape).astype(np.uint16)
