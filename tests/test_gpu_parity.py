@@ -493,3 +493,48 @@ def test_collaborative_step_equals_filter_then_prune_step(name):
             assert torch.equal(got["kidx"][b, : nk[b]], ref["kidx"][b, : nk[b]])
         for key in ("ho", "Ko", "Vo"):
             assert torch.equal(got[key].view(torch.int16), ref[key].view(torch.int16)), key
+
+
+def test_collaborative_step_replays_from_a_cuda_graph():
+    """The one-call step only enqueues work on the caller's stream (one memset, cooperative and programmatically
+    dependent launches): it can be captured once and replayed, with the same results as direct calls."""
+    w = W.workload("c0")
+    B, n = 2, w.Nv
+    feat = vb.bf16_tensor(W.make_features(w, B=B))
+    pos = torch.from_numpy(np.tile(W.make_positions(w), (B, 1, 1)).copy()).to(DEV)
+    K_b, V_b = W.make_kv(w, 0, n, B=B)
+    tK, tV = vb.bf16_tensor(K_b), vb.bf16_tensor(V_b)
+    th = vb.bf16_tensor(W.make_hidden(w, B=B))
+    budget, Ncap = w.budgets[-1], w.T + w.budgets[-1]
+    z = lambda *s, dt: torch.zeros(s, dtype=dt, device=DEV)
+
+    def outputs():
+        return dict(ho=z(B, Ncap, w.Dh, dt=torch.bfloat16), Ko=z(B, w.H, Ncap, w.d, dt=torch.bfloat16),
+                    Vo=z(B, w.H, Ncap, w.d, dt=torch.bfloat16), olen=z(B, dt=torch.int32),
+                    label=z(B, n, dt=torch.int32), ncl=z(B, dt=torch.int32))
+
+    def step(o, ws):
+        vb.vitcop_collaborative_step(feat, pos, th, tK, tV, w.vis_start, budget, o["ho"], o["Ko"], o["Vo"], o["olen"],
+                                     o["label"], o["ncl"], ws, metric=0, d_c=w.d_c, tau=w.tau, n_centers=w.n_centers)
+
+    ref, ws_ref = outputs(), vb.alloc_workspace(vb.OP_COLLAB_STEP, B=B, Nv=n, D=w.D)
+    step(ref, ws_ref)
+    torch.cuda.synchronize()
+    got, ws = outputs(), vb.alloc_workspace(vb.OP_COLLAB_STEP, B=B, Nv=n, D=w.D)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step(got, ws)                                     # warm-up outside the capture (function attributes, maps)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step(got, ws)
+    for _ in range(2):
+        for t in got.values():
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert vb.vitcop_poll_status(ws) == vb.OK
+        assert int(ref["olen"].min()) > w.T
+        for key in ("olen", "label", "ncl"):
+            assert torch.equal(got[key], ref[key]), key
+        for key in ("ho", "Ko", "Vo"):
+            assert torch.equal(got[key].view(torch.int16), ref[key].view(torch.int16)), key
