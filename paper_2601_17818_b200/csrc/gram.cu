@@ -173,6 +173,34 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// Two fp32 operations in one instruction (each half rounded like the scalar instruction): the epilogues are bound
+// by instruction issue, and a pair of neighbouring columns shares every step of the distance arithmetic.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float2 unpack2(unsigned long long v) {
+    float2 o;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(o.x), "=f"(o.y) : "l"(v));
+    return o;
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) wide,
 // laid out by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
@@ -400,6 +428,9 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
         rho_i = sm.rowrho[rl];
         if (SPATIAL) { x_i = sm.rowx[rl]; y_i = sm.rowy[rl]; }
     }
+    // the row's constants, twice each, for the paired arithmetic
+    const unsigned long long m2w2 = pack2(m2w_i, m2w_i), ai2 = pack2(a_i, a_i), two2 = pack2(2.f, 2.f);
+    const unsigned long long nxi2 = pack2(-x_i, -x_i), nyi2 = pack2(-y_i, -y_i), c22 = pack2(g.c2, g.c2);
     if (ok && call.wait_bar) ok = mbar_wait(call.wait_bar, call.wait_parity, call.abort_flag);
     ok = __all_sync(0xffffffffu, ok);
 
@@ -468,15 +499,30 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                     const float4 cw = cw4[q4];
                     float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (METRIC == 1) ca = ca4[q4];
-                    const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
-                    const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+                    if constexpr (GW == 32) {
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const int u = 4 * q4 + r;
-                        const float x = v[u] * cwv[r];
-                        const float base = METRIC == 0 ? 2.f : a_i + cav[r];
-                        const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
-                        v[u] = ex2_approx(d2 * g.c2);
+                        for (int h = 0; h < 2; ++h) {          // two neighbouring columns at a time
+                            const int u = 4 * q4 + 2 * h;
+                            const unsigned long long cw2 = h ? pack2(cw.z, cw.w) : pack2(cw.x, cw.y);
+                            const unsigned long long ca2 = h ? pack2(ca.z, ca.w) : pack2(ca.x, ca.y);
+                            const unsigned long long x2 = mul2(pack2(v[u], v[u + 1]), cw2);
+                            const unsigned long long base2 = METRIC == 0 ? two2 : add2(ai2, ca2);
+                            const float2 d2 = unpack2(fma2(x2, m2w2, base2));
+                            const float2 arg = unpack2(mul2(pack2(fmaxf(d2.x, 0.f), fmaxf(d2.y, 0.f)), c22));
+                            v[u] = ex2_approx(arg.x);
+                            v[u + 1] = ex2_approx(arg.y);
+                        }
+                    } else {
+                        const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                        const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            const int u = 4 * q4 + r;
+                            const float x = v[u] * cwv[r];
+                            const float base = METRIC == 0 ? 2.f : a_i + cav[r];
+                            const float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                            v[u] = ex2_approx(d2 * g.c2);
+                        }
                     }
                 }
                 if (!full) {
@@ -502,22 +548,48 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                     float4 ca = make_float4(0.f, 0.f, 0.f, 0.f), cx = ca, cy = ca;
                     if (METRIC == 1) ca = ca4[q4];
                     if (SPATIAL) { cx = cx4[q4]; cy = cy4[q4]; }
-                    const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
                     const float crv[4] = {cr.x, cr.y, cr.z, cr.w};
-                    const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
-                    const float cxv[4] = {cx.x, cx.y, cx.z, cx.w};
-                    const float cyv[4] = {cy.x, cy.y, cy.z, cy.w};
+                    float d2v[4], s2v[4];              // squared feature distance (unclamped), squared spatial distance
+                    if constexpr (GW == 32) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {          // two neighbouring columns at a time
+                            const int u = 4 * q4 + 2 * h;
+                            const unsigned long long cw2 = h ? pack2(cw.z, cw.w) : pack2(cw.x, cw.y);
+                            const unsigned long long ca2 = h ? pack2(ca.z, ca.w) : pack2(ca.x, ca.y);
+                            const unsigned long long x2 = mul2(pack2(v[u], v[u + 1]), cw2);
+                            const unsigned long long base2 = METRIC == 0 ? two2 : add2(ai2, ca2);
+                            const float2 d2 = unpack2(fma2(x2, m2w2, base2));
+                            d2v[2 * h] = d2.x;
+                            d2v[2 * h + 1] = d2.y;
+                            if (SPATIAL) {
+                                const unsigned long long dx2 = add2(h ? pack2(cx.z, cx.w) : pack2(cx.x, cx.y), nxi2);
+                                const unsigned long long dy2 = add2(h ? pack2(cy.z, cy.w) : pack2(cy.x, cy.y), nyi2);
+                                const float2 s2 = unpack2(fma2(dx2, dx2, mul2(dy2, dy2)));
+                                s2v[2 * h] = s2.x;
+                                s2v[2 * h + 1] = s2.y;
+                            }
+                        }
+                    } else {
+                        const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                        const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+                        const float cxv[4] = {cx.x, cx.y, cx.z, cx.w};
+                        const float cyv[4] = {cy.x, cy.y, cy.z, cy.w};
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            const float x = v[4 * q4 + r] * cwv[r];
+                            d2v[r] = fmaf(x, m2w_i, METRIC == 0 ? 2.f : a_i + cav[r]);
+                            if (SPATIAL) {
+                                const float dx = cxv[r] - x_i, dy = cyv[r] - y_i;
+                                s2v[r] = fmaf(dx, dx, dy * dy);
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int r = 0; r < 4; ++r) {
                         const int u = 4 * q4 + r;
-                        const float x = v[u] * cwv[r];
-                        const float base = METRIC == 0 ? 2.f : a_i + cav[r];
-                        float d2 = fmaxf(fmaf(x, m2w_i, base), 0.f);
+                        float d2 = fmaxf(d2v[r], 0.f);
                         bool usable = true;        // the pair may serve as (child, parent) at all
-                        if (SPATIAL) {
-                            const float dx = cxv[r] - x_i, dy = cyv[r] - y_i;
-                            usable = fmaf(dx, dx, dy * dy) <= g.tau2;
-                        }
+                        if (SPATIAL) usable = s2v[r] <= g.tau2;
                         if (!full) {
                             const int j = J0 + cl0 + u;
                             usable = usable && j > i && j < g.n && row_valid;
