@@ -14,16 +14,19 @@ __device__ __forceinline__ uint4 knorm_ld_stream(const uint4* p) {
     return v;
 }
 
+// a0 += (low halves)^2, a1 += (high halves)^2 of the four bf16 pairs, pair by pair: the two accumulators advance
+// together as one fp32x2 fused multiply-add per pair (each half rounded like the scalar instruction).
 __device__ __forceinline__ void knorm_sq_acc(const uint4& v, float& a0, float& a1) {
-    float x;
-    x = bf16lo(v.x); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.x); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.y); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.y); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.z); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.z); a1 = fmaf(x, x, a1);
-    x = bf16lo(v.w); a0 = fmaf(x, x, a0);
-    x = bf16hi(v.w); a1 = fmaf(x, x, a1);
+    unsigned long long acc;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(acc) : "f"(a0), "f"(a1));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        unsigned long long x;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "r"(w[q] << 16), "r"(w[q] & 0xffff0000u));
+        asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(x));
+    }
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc));
 }
 
 // Sum of squares of the 16-byte pieces sub, sub + LPR, ... of one token's K rows over all H heads (`base` points at
