@@ -11,6 +11,8 @@
 //                             inside the spatial radius (Eq. 3) as a packed (d^2, j) 64-bit minimum
 //   5. vic_finalize_kernel    gamma = rho * delta, radix-select of the centres, pointer jumping over the
 //                             parent forest, orphan fallback, labels (Algorithm 2, steps 3-4)
+// Small problems replace 1-4 by gram_resident_kernel (gram.cu): one pass over the Gram tiles, accumulators kept in
+// tensor memory.
 #include "gram.cuh"
 
 namespace vitcop {

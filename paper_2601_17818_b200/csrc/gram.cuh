@@ -89,8 +89,9 @@ __host__ __device__ inline float rho_from_partials(const float* p, const GramTil
     return s;
 }
 
-// True when the whole symmetric sweep of the problem fits the tensor memory of one wave of CTAs (at most four
-// 128 x 128 tiles per SM): density and delta can then share one pass over the Gram tiles (launch_gram_resident).
+// True when the whole symmetric sweep of the problem fits the tensor memory of one wave of CTAs (at most two units
+// of one row block against two column blocks per SM): density and delta can then share one pass over the Gram tiles
+// (launch_gram_resident).
 bool gram_fits_resident(int B, int n);
 
 // True when the resident sweep can compute the K-norm of keys with H heads of d elements on the side.
