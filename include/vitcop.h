@@ -72,6 +72,18 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
  * workspace resets the word when it starts, so poll after the call of interest. */
 int vitcop_poll_status(const void* workspace, void* stream, int* device_status);
 
+/* ---------------------------------------------------------------- diagnostic: bounded device waits
+ * The paper has no counterpart.  Kernels whose CTAs wait for one another or for asynchronous copies (the Gram
+ * sweeps of the redundancy filter) bound every wait; when a wait runs out, the CTA abandons its work, lets its
+ * copies and tensor-core operations in flight finish, frees its tensor memory and records VITCOP_ERR_TIMEOUT in
+ * the status word (read it with vitcop_poll_status; the call's outputs are then undefined, the workspace and the
+ * library remain usable).  This call sets the limit for launches made after it, process-wide:
+ *   limit_ns      time after which a wait gives up; 0 restores the default of 2 s
+ *   expire_roles  for failure-handling tests: waits of the named roles give up at once, whatever their state
+ *                 (1 load warp, 2 tensor-core issue warp, 4 epilogue warps; 0 = none)
+ * Always returns VITCOP_OK. */
+int vitcop_set_wait_limit(unsigned long long limit_ns, int expire_roles);
+
 /* ---------------------------------------------------------------- diagnostic: per-kernel device times
  * The paper has no counterpart; this exists so that a benchmark can attribute the time of a multi-kernel
  * call to its kernels.  Between vitcop_kernel_timing_begin and vitcop_kernel_timing_end every kernel the
@@ -227,6 +239,7 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V,
  *   feat bf16 [B, Nv, D], pos fp32 [B, Nv, 2] or NULL, fp (host) as in vitcop_redundancy_filter
  *   hidden, K, V, the outputs, kept_pos, out_len as in vitcop_prune_step (Nv_cap = Nv)
  *   label_out int32 [B, Nv] and n_clusters_out int32 [B]: required outputs (the labels the selection used)
+ *   rho_out, delta2_out fp32 [B, Nv], parent_out int32 [B, Nv]: optional, as in vitcop_redundancy_filter
  *   score_out, keep_idx_out [B, Nv], n_keep_out [B]: optional
  *   workspace: vitcop_workspace_bytes(VITCOP_OP_COLLAB_STEP, B, 0, 0, 0, Nv, D, 0) bytes; one status word
  * Errors: as the two calls it replaces. */
@@ -236,6 +249,7 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
                               void* hidden_out, void* K_out, void* V_out, int Ncap,
                               int32_t* kept_pos, int32_t* out_len,
                               int32_t* label_out, int32_t* n_clusters_out,
+                              float* rho_out, float* delta2_out, int32_t* parent_out,
                               float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out,
                               void* workspace, size_t workspace_bytes, void* stream);
 

@@ -12,7 +12,7 @@
 //     no sum is split, blocked or reordered by it.
 //   * all functions are per call stateless; outputs are caller-allocated.
 //
-// Readings of the paper adopted where it is silent (each also listed in the design notes):
+// Readings of the paper adopted where it is silent:
 //   R1  density order is total: j is "denser" than i iff rho_j > rho_i, or rho_j == rho_i and j < i
 //       (Eq. 3 / Algorithm 2 step 2 print a strict ">" which leaves exact duplicates unordered).
 //   R2  a token with no admissible denser neighbour ("orphan", delta = +inf, N_i = -1) ranks first
@@ -174,7 +174,6 @@ void oracle_feature_distance_rows(const uint16_t* feat, int n, int D, int metric
         for (int j = 0; j < n; ++j) {
             const float* c = &f[static_cast<size_t>(j) * D];
             double g = 0.0;
-#pragma omp simd reduction(+ : g)
             for (int e = 0; e < D; ++e) g += static_cast<double>(a[e]) * static_cast<double>(c[e]);
             double s, dist2;
             if (metric == 0) {

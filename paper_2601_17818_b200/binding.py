@@ -27,7 +27,7 @@ EXPORTS = [
     "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
     "vitcop_prune_step_static", "vitcop_merge_clusters", "vitcop_cls_saliency", "vitcop_stage_count",
     "vitcop_flops_layer", "vitcop_visual_tokens_at_layer", "vitcop_flops_total", "vitcop_cr_int",
-    "vitcop_collaborative_step",
+    "vitcop_collaborative_step", "vitcop_set_wait_limit",
 ]
 
 
@@ -94,8 +94,9 @@ def lib() -> C.CDLL:
         L.vitcop_cr_int.argtypes = [f64, f64, f64, i32, i32, i32]
         L.vitcop_cr_int.restype = f64
         L.vitcop_collaborative_step.argtypes = [vp, vp, i32, C.POINTER(FilterParams), vp, vp, vp, i32, i32, i32, i32,
-                                                i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz,
-                                                vp]
+                                                i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                vp, vp, sz, vp]
+        L.vitcop_set_wait_limit.argtypes = [C.c_ulonglong, i32]
         L.vitcop_kernel_timing_begin.argtypes = []
         L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
@@ -232,7 +233,7 @@ def vitcop_prune_step_static(hidden, K, V, vis_start: int, vis_len, Nv_cap: int,
 def vitcop_collaborative_step(feat, pos, hidden, K, V, vis_start: int, budget: int, hidden_out, K_out, V_out, out_len,
                               label_out, n_clusters_out, workspace, metric: int = 0, d_c: float = 0.5, tau: float = 0.6,
                               alpha: float = 0.05, n_centers: int = 0, kept_pos=None, score_out=None, keep_idx_out=None,
-                              n_keep_out=None):
+                              n_keep_out=None, rho=None, delta2=None, parent=None):
     """Stage II in one call: redundancy filter + fused pruning step in quota mode, K-norm beside the clustering."""
     B, Nv, D = feat.shape
     _, H, N, d = K.shape
@@ -242,7 +243,7 @@ def vitcop_collaborative_step(feat, pos, hidden, K, V, vis_start: int, budget: i
     rc = lib().vitcop_collaborative_step(_ptr(feat), _ptr(pos), D, C.byref(p), _ptr(hidden), _ptr(K), _ptr(V), B, H, N,
                                          d, Dh, vis_start, Nv, int(budget), _ptr(hidden_out), _ptr(K_out), _ptr(V_out),
                                          Ncap, _ptr(kept_pos), _ptr(out_len), _ptr(label_out), _ptr(n_clusters_out),
-                                         _ptr(score_out), _ptr(keep_idx_out), _ptr(n_keep_out), _ptr(workspace),
+                                         _ptr(rho), _ptr(delta2), _ptr(parent), _ptr(score_out), _ptr(keep_idx_out), _ptr(n_keep_out), _ptr(workspace),
                                          workspace.numel(), _stream())
     _check(rc, "vitcop_collaborative_step")
     return out_len
@@ -315,6 +316,11 @@ def vitcop_similarity_rows(feat: torch.Tensor, metric: int, row_begin: int, row_
                                       _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "vitcop_similarity_rows")
     return out
+
+
+def vitcop_set_wait_limit(limit_ns: int = 0, expire_roles: int = 0) -> None:
+    """Limit of the kernels' bounded waits (0 = default 2 s); ``expire_roles`` makes the named roles give up at once."""
+    _check(lib().vitcop_set_wait_limit(int(limit_ns), int(expire_roles)), "vitcop_set_wait_limit")
 
 
 def vitcop_kernel_timing_begin() -> None:

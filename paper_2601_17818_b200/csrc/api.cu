@@ -6,6 +6,7 @@
 #include <mutex>
 #include <vector>
 
+#include "gram.cuh"
 #include "internal.cuh"
 
 namespace vitcop {
@@ -142,6 +143,11 @@ const char* vitcop_status_string(int status) {
 }
 
 int vitcop_last_cuda_error(void) { return g_last_cuda_error; }
+
+int vitcop_set_wait_limit(unsigned long long limit_ns, int expire_roles) {
+    gram_set_wait_debug(limit_ns, expire_roles);
+    return VITCOP_OK;
+}
 
 int vitcop_kernel_timing_begin(void) {
     std::lock_guard<std::mutex> lock(g_timing_mutex);
@@ -309,11 +315,16 @@ int vitcop_prune_step(const void* hidden, const void* K, const void* V, int B, i
     int32_t* nkeep = n_keep_out ? n_keep_out : reinterpret_cast<int32_t*>(ws + lay.off_nkeep);
     rc = reset_status(workspace, s);
     if (rc != VITCOP_OK) return rc;
+    bool have_knorm = false;
     rc = launch_knorm(K, B, H, d, (int64_t)H * N * d, (int64_t)N * d, d, vis_start, vis_len, vis_len_uniform, score,
-                      Nv_cap, s);
+                      Nv_cap, s, false, &have_knorm);
     if (rc != VITCOP_OK) return rc;
+    // The selection releases its dependents before it waits for its predecessor, and the compaction copies the rows
+    // in front of the span before its own wait: that is safe only behind a kernel of this call that has itself
+    // waited for everything queued before the call.  With an empty span there is no such kernel, so the selection
+    // is then launched in plain stream order.
     rc = launch_select(score, label, B, vis_len, vis_len_uniform, Nv_cap, label ? 1 : 0, 0, budget, keep, Nv_cap,
-                       nkeep, nullptr, reinterpret_cast<int*>(ws), s, true);
+                       nkeep, nullptr, reinterpret_cast<int*>(ws), s, have_knorm);
     if (rc != VITCOP_OK) return rc;
     return launch_compact(hidden, K, V, B, H, N, d, Dh, seq_len, vis_start, vis_len, vis_len_uniform, keep, Nv_cap,
                           nkeep, hidden_out, K_out, V_out, Ncap, kept_pos, out_len, s, true);
@@ -323,8 +334,9 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
                               const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,
                               int vis_start, int Nv, int budget, void* hidden_out, void* K_out, void* V_out, int Ncap,
                               int32_t* kept_pos, int32_t* out_len, int32_t* label_out, int32_t* n_clusters_out,
-                              float* score_out, int32_t* keep_idx_out, int32_t* n_keep_out, void* workspace,
-                              size_t workspace_bytes, void* stream) {
+                              float* rho_out, float* delta2_out, int32_t* parent_out, float* score_out,
+                              int32_t* keep_idx_out, int32_t* n_keep_out, void* workspace, size_t workspace_bytes,
+                              void* stream) {
     if (!feat || !fp || !K || !out_len || !label_out || !n_clusters_out || budget < 0 || Nv < 0 || D < 0)
         return VITCOP_ERR_INVALID_ARG;
     if (fp->metric != 0 && fp->metric != 1) return VITCOP_ERR_INVALID_ARG;
@@ -333,7 +345,8 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
     if (rc != VITCOP_OK) return rc;
     rc = check_span(N, vis_start, nullptr, Nv, Nv);
     if (rc != VITCOP_OK) return rc;
-    if (D % 64 || !aligned16(feat) || !aligned8(pos) || Nv > VITCOP_MAX_VISUAL_TOKENS) return VITCOP_ERR_UNSUPPORTED;
+    if (D % 64 || !aligned16(feat) || !aligned8(pos) || Nv > VITCOP_MAX_VISUAL_TOKENS || B > 65535)
+        return VITCOP_ERR_UNSUPPORTED;
     const size_t filter_bytes = align_up(filter_workspace_bytes(B, Nv, D), 256);
     const StepWs lay(B, Nv);
     if (!workspace || workspace_bytes < filter_bytes + lay.total || !aligned256(workspace)) return VITCOP_ERR_WORKSPACE;
@@ -354,12 +367,13 @@ int vitcop_collaborative_step(const void* feat, const float* pos, int D, const v
     if (B == 0) return VITCOP_OK;
     if (Nv > 0) {
         const KnormJob job = {K, B, H, N, d, vis_start, Nv, score};
-        rc = launch_filter(feat, pos, B, Nv, D, *fp, nc, label_out, n_clusters_out, nullptr, nullptr, nullptr, workspace,
-                           s, &job);
+        rc = launch_filter(feat, pos, B, Nv, D, *fp, nc, label_out, n_clusters_out, rho_out, delta2_out, parent_out,
+                           workspace, s, &job);
         if (rc != VITCOP_OK) return rc;
     }
+    // (plain stream order when the filter was skipped: see vitcop_prune_step)
     rc = launch_select(score, label_out, B, nullptr, Nv, Nv, 1, 0, budget, keep, Nv, nkeep, nullptr,
-                       reinterpret_cast<int*>(ws), s, true);
+                       reinterpret_cast<int*>(ws), s, Nv > 0);
     if (rc != VITCOP_OK) return rc;
     return launch_compact(hidden, K, V, B, H, N, d, Dh, nullptr, vis_start, nullptr, Nv, keep, Nv, nkeep, hidden_out,
                           K_out, V_out, Ncap, kept_pos, out_len, s, true);

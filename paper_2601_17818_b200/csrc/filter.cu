@@ -18,8 +18,6 @@
 namespace vitcop {
 namespace {
 
-constexpr int BM = kGramBM;
-
 // ------------------------------------------------------------------------------------------------
 // small kernels
 // ------------------------------------------------------------------------------------------------
@@ -42,24 +40,6 @@ __global__ void rho_reduce_kernel(const float* __restrict__ part, int n, GramTil
 // Centres, forest roots and labels: one CTA per sample.
 // ------------------------------------------------------------------------------------------------
 constexpr int kFinThreads = 1024;
-
-__device__ __forceinline__ uint32_t fin_prefix_count(bool flag, uint32_t* warp_sums, uint32_t& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bal = __ballot_sync(0xffffffffu, flag);
-    const uint32_t before = __popc(bal & ((1u << lane) - 1u));
-    if (lane == 0) warp_sums[warp] = __popc(bal);
-    __syncthreads();
-    uint32_t v = warp_sums[lane];
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
-    }
-    total = __shfl_sync(0xffffffffu, v, 31);
-    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
-    __syncthreads();
-    return (warp == 0 ? 0u : base) + before;
-}
 
 // Shared memory: keys[n] (uint64; later reused as next[n] int32), isc[n] (uint8), centres[nc] (int32).
 __global__ void __launch_bounds__(kFinThreads)
@@ -174,12 +154,12 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
             else {
                 const bool eq = i < n && key == T;
                 uint32_t eq_total;
-                const uint32_t eq_rank = eq_running + fin_prefix_count(eq, warp_sums, eq_total);
+                const uint32_t eq_rank = eq_running + block_prefix_count(eq, warp_sums, eq_total);
                 eq_running += eq_total;
                 f = i < n && (key < T || (eq && eq_rank < krem));
             }
             uint32_t c_total;
-            const uint32_t r = c_running + fin_prefix_count(f, warp_sums, c_total);
+            const uint32_t r = c_running + block_prefix_count(f, warp_sums, c_total);
             c_running += c_total;
             if (i < n) isc[i] = f ? 1 : 0;
             if (f && r < (uint32_t)nc) centres[r] = i;

@@ -20,6 +20,8 @@
 // VITCOP_ERR_TIMEOUT is written to the status word.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "gram.cuh"
 #include "knorm.cuh"
 
@@ -33,7 +35,7 @@ constexpr int UMMA_K = 16;
 // TMEM lane quarter).  The delta sweep's epilogue is the heavier one and gets twice the warps.
 __host__ __device__ constexpr int epi_slices(int mode) { return mode == GRAM_DELTA ? 4 : 2; }
 __host__ __device__ constexpr int gemm_threads(int mode) { return 64 + epi_slices(mode) * 128; }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s give up and leave
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s (default) give up and leave
 constexpr unsigned long long kDrainLimitNs = 20000000ull;    // bounded waits for this CTA's own copies / MMAs after giving up
 
 // ------------------------------------------------------------------------------------------------
@@ -67,14 +69,19 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // Bounded wait.  Returns false (after raising `abort_flag`) when the time limit is hit or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
+// limit_ns == 0 gives up at once, whatever the barrier's state (failure-handling tests use it to send one role of
+// a CTA down the give-up path while the others have work in flight).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
+    if (limit_ns != 0ull) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) break;
+        const unsigned long long t0 = global_ns();
+        for (uint32_t it = 1;; ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((it & 63u) == 0u) {
+                if (*abort_flag) return false;
+                if (global_ns() - t0 > limit_ns) break;
+            }
         }
     }
     *abort_flag = 1;
@@ -224,7 +231,13 @@ struct KernelArgs {
     GramTiling t;
     long long total_tiles;         // the resident sweep counts its units here
     int extra_units_per_b;         // resident sweep: units of one sample that do not hold a diagonal tile
+    unsigned long long wait_ns;    // time limit of every bounded wait
+    int expire_roles;              // roles whose waits give up at once: 1 load warp, 2 MMA warp, 4 epilogue warps
+    __device__ __forceinline__ unsigned long long limit_of(int role) const {
+        return (expire_roles & role) ? 0ull : wait_ns;
+    }
 };
+constexpr int kRoleLoad = 1, kRoleMma = 2, kRoleEpi = 4;
 
 template <int BN, bool SYM, bool DIAG = false>
 __device__ __forceinline__ void decode_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
@@ -336,6 +349,7 @@ struct EpiCall {
     uint32_t arrive_bar;           // mbarrier to arrive on once this thread has read the accumulator (0: none)
     bool rho_from_part;            // GRAM_DELTA: sum rho from the density partials (and publish it from diagonal tiles)
     volatile int* abort_flag;
+    unsigned long long limit_ns;   // time limit of the wait for the accumulator
 };
 
 // Returns true when the CTA must give up (a bounded wait expired somewhere).
@@ -431,7 +445,7 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
     // the row's constants, twice each, for the paired arithmetic
     const unsigned long long m2w2 = pack2(m2w_i, m2w_i), ai2 = pack2(a_i, a_i), two2 = pack2(2.f, 2.f);
     const unsigned long long nxi2 = pack2(-x_i, -x_i), nyi2 = pack2(-y_i, -y_i), c22 = pack2(g.c2, g.c2);
-    if (ok && call.wait_bar) ok = mbar_wait(call.wait_bar, call.wait_parity, call.abort_flag);
+    if (ok && call.wait_bar) ok = mbar_wait(call.wait_bar, call.wait_parity, call.abort_flag, call.limit_ns);
     ok = __all_sync(0xffffffffu, ok);
 
     float racc = 0.f;                              // GRAM_RHO: row-side sum
@@ -740,21 +754,22 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const long long total_tiles = k.total_tiles;
     const int KB = g.D / BK;
+    uint32_t issued = 0, issued_parity = 0;    // thread 0, per stage: a load was issued / parity of its phase
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         // The features are an input of the whole call (never written by the kernel before this one), so
         // the loads need not wait for the preceding grid.
         if (lane == 0) {
+            const unsigned long long lim = k.limit_of(kRoleLoad);
             uint32_t stage = 0, phase = 0;
-            uint32_t issued = 0, issued_parity = 0;        // per stage: a load was issued / parity of its phase
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
                 int b, ti, tj;
                 decode_tile<BN, SYM, DIAG>(k, t, b, ti, tj);
                 const int I0 = g.row0 + ti * BM, J0 = tj * BN;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, lim)) { ok = false; break; }
                     const uint32_t sa = tiles + stage * S::kStageBytes;
                     mbar_expect_tx(bar_full + 8 * stage, DIAG ? S::kABytes : S::kStageBytes);
                     tma_load_3d(sa, &map_a, bar_full + 8 * stage, kb * BK, I0, b);
@@ -764,25 +779,21 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                // leaving early: give the copies still in flight into this CTA's shared memory time to land
-                for (int s = 0; s < S::kStages; ++s)
-                    if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
-            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            const unsigned long long lim = k.limit_of(kRoleMma);
             uint32_t stage = 0, phase = 0;
             uint32_t acc = 0, acc_phase = 0;
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abort_flag, lim)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, lim)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles + stage * S::kStageBytes;
                     const uint64_t da = umma_desc_k128(sa), db = DIAG ? da : umma_desc_k128(sa + S::kABytes);
@@ -821,6 +832,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             c.arrive_bar = bar_tempty + 8 * acc;
             c.rho_from_part = false;
             c.abort_flag = abort_flag;
+            c.limit_ns = k.limit_of(kRoleEpi);
             if (epi_tile<BN, MODE, METRIC, SPATIAL, NS>(k, sm, c, ok)) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
@@ -832,7 +844,13 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (threadIdx.x == 0 && *abort_flag && g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag) {
+        // Some role gave up, so loads this thread issued may never have been consumed: give the copies still in
+        // flight into this CTA's shared memory time to land before the CTA goes away.
+        for (int s = 0; s < S::kStages; ++s)
+            if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
+        if (g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+    }
 }
 
 
@@ -872,14 +890,15 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
 // Barrier over all CTAs of the grid, called by the epilogue threads.  Returns true when the grid must give up.
 // One thread speaks for the CTA: the CTA barrier orders every epilogue thread's writes before that thread's fence
 // (and its fence before their later reads), so the other threads need none of their own.
-__device__ __forceinline__ bool resident_grid_barrier(unsigned int* counter, volatile int* abort_flag, bool aborted) {
+__device__ __forceinline__ bool resident_grid_barrier(unsigned int* counter, volatile int* abort_flag, bool aborted,
+                                                      unsigned long long limit_ns) {
     epi_bar_sync<kResidentEpiThreads>();
     if (threadIdx.x == 64 && !aborted) {
         __threadfence();
         atomicAdd(counter, 1u);
         const unsigned long long t0 = global_ns();
         while (ld_acquire_u32(counter) < gridDim.x) {
-            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+            if (limit_ns == 0ull || global_ns() - t0 > limit_ns) { *abort_flag = 1; break; }
         }
         __threadfence();
     }
@@ -897,11 +916,11 @@ __device__ __forceinline__ void resident_publish(unsigned int* flag) {
 
 // Waits (bounded) until both flags are up.  Returns true when the grid must give up.
 __device__ __forceinline__ bool resident_wait_flags(const unsigned int* fa, const unsigned int* fb,
-                                                    volatile int* abort_flag, bool aborted) {
+                                                    volatile int* abort_flag, bool aborted, unsigned long long limit_ns) {
     if (threadIdx.x == 64 && !aborted) {
         const unsigned long long t0 = global_ns();
         while (ld_acquire_u32(fa) == 0u || ld_acquire_u32(fb) == 0u) {
-            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+            if (limit_ns == 0ull || global_ns() - t0 > limit_ns) { *abort_flag = 1; break; }
         }
         __threadfence();
     }
@@ -958,7 +977,7 @@ constexpr int kKnBuffers = 3;
 // of the sixteen-lane reduction of the stand-alone kernel, so that both give the same bits.
 __device__ __forceinline__ void resident_knorm(const GramArgs& g, const uint8_t* buf_gen, uint32_t buf_smem,
                                                uint32_t buf_bytes, uint32_t bar_kn, uint32_t bar_last_mma,
-                                               volatile int* abort_flag) {
+                                               volatile int* abort_flag, unsigned long long limit_ns) {
     const int tid = threadIdx.x;                           // 0 .. 63
     auto all_ok = [](bool ok) {
         uint32_t out;
@@ -971,7 +990,7 @@ __device__ __forceinline__ void resident_knorm(const GramArgs& g, const uint8_t*
         return out != 0;
     };
     // the tensor cores read the operand buffers until the last MMA completes
-    if (!all_ok(mbar_wait(bar_last_mma, 0, abort_flag))) return;
+    if (!all_ok(mbar_wait(bar_last_mma, 0, abort_flag, limit_ns))) return;
 
     const int H = g.kn_H, d8 = g.kn_d / 8, Nv = g.kn_Nv;
     const uint32_t row_bytes = (uint32_t)d8 * 16u;
@@ -1003,7 +1022,7 @@ __device__ __forceinline__ void resident_knorm(const GramArgs& g, const uint8_t*
     bool ok = true;
     for (long long c = blockIdx.x; c < total; c += gridDim.x, ++it) {
         const int buf = (int)(it % nbuf);
-        ok = all_ok(mbar_wait(bar_kn + 8 * buf, (uint32_t)((it / nbuf) & 1), abort_flag));
+        ok = all_ok(mbar_wait(bar_kn + 8 * buf, (uint32_t)((it / nbuf) & 1), abort_flag, limit_ns));
         if (!ok) break;
         const int b = (int)(c / chunks_per_b);
         const int i0 = (int)(c - (long long)b * chunks_per_b) * kKnChunkTokens;
@@ -1090,18 +1109,19 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
     const long long total_units = k.total_tiles;          // <= kResidentUnits * gridDim.x (checked by the launcher)
     const int KB = g.D / BK;
+    uint32_t issued = 0, issued_parity = 0;               // thread 0, per stage: a load was issued / parity of its phase
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            const unsigned long long lim = k.limit_of(kRoleLoad);
             uint32_t stage = 0, phase = 0;
-            uint32_t issued = 0, issued_parity = 0;
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_units; t += gridDim.x) {
                 const ResidentUnit u = decode_resident_unit(k, t);
                 const int I0 = u.ti * BM, J0 = u.tj0 * BM;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, lim)) { ok = false; break; }
                     const uint32_t sa = tiles + stage * S::kStageBytes;
                     // rows of the box past the sample's last token are zero-filled and still count as received
                     mbar_expect_tx(bar_full + 8 * stage, S::kStageBytes);
@@ -1112,22 +1132,19 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                for (int s = 0; s < S::kStages; ++s)
-                    if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
-            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer: unit s of this CTA -> columns 256 s ..
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(BM, kResidentBN);
+            const unsigned long long lim = k.limit_of(kRoleMma);
             uint32_t stage = 0, phase = 0;
             uint32_t slot = 0;
             bool ok = true;
             for (long long t = blockIdx.x; ok && t < total_units; t += gridDim.x, ++slot) {
                 const uint32_t d_tmem = tmem_base + slot * kResidentBN;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, lim)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles + stage * S::kStageBytes;
                     const uint64_t da = umma_desc_k128(sa), db = umma_desc_k128(sa + S::kABytes);
@@ -1152,12 +1169,13 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (g.kn_K) {
             const long long my_units = (total_units - blockIdx.x + gridDim.x - 1) / gridDim.x;   // >= 1
             resident_knorm(g, gen, tiles, (uint32_t)S::kTileBytes, bar_kn, bar_tfull + 8 * (uint32_t)(my_units - 1),
-                           abort_flag);
+                           abort_flag, k.limit_of(kRoleLoad | kRoleMma));
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..17)
         bool ok = true;
         bool stop = false;
+        const unsigned long long lim = k.limit_of(kRoleEpi);
         grid_dependency_wait();
         // tile s (0 or 1) of this CTA's unit number `slot`
         auto tile_call = [&](const ResidentUnit& u, uint32_t slot, int s, bool wait_mma, bool rho_from_part) {
@@ -1171,6 +1189,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             c.arrive_bar = 0;
             c.rho_from_part = rho_from_part;
             c.abort_flag = abort_flag;
+            c.limit_ns = lim;
             return c;
         };
 
@@ -1191,11 +1210,11 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const EpiCall c = tile_call(u, slot, s, true, false);
                 if (c.ti != c.tj)
                     stop = resident_wait_flags(g.diag_ready + (size_t)c.b * k.t.TI + c.ti,
-                                               g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop);
+                                               g.diag_ready + (size_t)c.b * k.t.TI + c.tj, abort_flag, stop, lim);
                 if (!stop) stop = epi_tile<BN, GRAM_RHO, METRIC, false, NS, 8>(k, sm, c, ok);
             }
         }
-        stop = resident_grid_barrier(g.grid_sync, abort_flag, stop);
+        stop = resident_grid_barrier(g.grid_sync, abort_flag, stop, lim);
         // The kernels that follow cannot share an SM with a CTA of this grid (registers, shared memory); from here
         // on they may at least be set up.
         grid_dependency_launch_dependents();
@@ -1217,7 +1236,12 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (threadIdx.x == 0 && *abort_flag && g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag) {
+        // (see gram_tc_kernel: unconsumed operand loads must have landed before the CTA goes away)
+        for (int s = 0; s < S::kStages; ++s)
+            if (issued >> s & 1u) mbar_drain(bar_full + 8 * s, issued_parity >> s & 1u);
+        if (g.status) atomicMax(g.status, VITCOP_ERR_TIMEOUT);
+    }
     grid_dependency_launch_dependents();
 }
 
@@ -1255,26 +1279,46 @@ bool make_feat_map(CUtensorMap* map, const void* feat, int B, int n, int D, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Time limit of the kernels' bounded waits and, for failure-handling tests, the roles whose waits give up at once.
+std::atomic<unsigned long long> g_wait_ns{kWaitLimitNs};
+std::atomic<int> g_expire_roles{0};
+
+// What the launchers remember is remembered per device: one process may drive several.
+constexpr int kMaxDevices = 64;
+int current_device() {
+    int dev = 0;
+    return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) ? dev : 0;
+}
+
 int num_sms() {
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    static std::atomic<int> sms[kMaxDevices];
+    const int dev = current_device();
+    int v = sms[dev].load(std::memory_order_relaxed);
+    if (v <= 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        sms[dev].store(v, std::memory_order_relaxed);
     }
-    return sms;
+    return v;
+}
+
+// Raises a kernel's dynamic shared-memory limit once per device.
+template <typename Kernel>
+int allow_dynamic_smem(Kernel kern, int bytes, std::atomic<unsigned long long>& done) {
+    const unsigned long long bit = 1ull << current_device();
+    if (done.load(std::memory_order_relaxed) & bit) return VITCOP_OK;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return record_cuda(e);
+    done.fetch_or(bit, std::memory_order_relaxed);
+    return VITCOP_OK;
 }
 
 template <int BN, int MODE, int METRIC, bool SPATIAL>
 int launch_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream, bool pdl) {
     using S = GemmSmem<BN>;
-    static bool attr_done = false;
+    static std::atomic<unsigned long long> attr_done{0};
     auto kern = gram_tc_kernel<BN, MODE, METRIC, SPATIAL>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal);
-        if (e != cudaSuccess) return record_cuda(e);
-        attr_done = true;
-    }
+    const int arc = allow_dynamic_smem(kern, S::kTotal, attr_done);
+    if (arc != VITCOP_OK) return arc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(k.total_tiles < num_sms() ? k.total_tiles : num_sms()));
     cfg.blockDim = dim3(gemm_threads(MODE));
@@ -1321,13 +1365,10 @@ int launch_bn(int mode, const CUtensorMap& ma, const CUtensorMap& mb, const Kern
 template <int METRIC, bool SPATIAL>
 int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const KernelArgs& k, cudaStream_t stream) {
     using S = GemmSmem<kResidentBN>;
-    static bool attr_done = false;
+    static std::atomic<unsigned long long> attr_done{0};
     auto kern = gram_resident_kernel<METRIC, SPATIAL>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal);
-        if (e != cudaSuccess) return record_cuda(e);
-        attr_done = true;
-    }
+    const int arc = allow_dynamic_smem(kern, S::kTotal, attr_done);
+    if (arc != VITCOP_OK) return arc;
     const long long ctas = (k.total_tiles + kResidentUnits - 1) / kResidentUnits;
     cudaLaunchConfig_t cfg = {};
     // as many CTAs as there are SMs (never fewer than the units need): the shortest chain of units per CTA
@@ -1345,6 +1386,11 @@ int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const Kern
 }
 
 }  // namespace
+
+void gram_set_wait_debug(unsigned long long limit_ns, int expire_roles) {
+    g_wait_ns.store(limit_ns ? limit_ns : kWaitLimitNs);
+    g_expire_roles.store(expire_roles & 7);
+}
 
 int gram_pick_bn(int B, int n) {
     const long long ti = (n + BM - 1) / BM;
@@ -1369,6 +1415,9 @@ int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const Gr
         if (mode == GRAM_DIAG) k.t.tiles_per_b = k.t.TI;        // one tile per 128-row block (tiling.BN == 128)
     }
     k.total_tiles = (long long)args.B * k.t.tiles_per_b;
+    k.extra_units_per_b = 0;
+    k.wait_ns = g_wait_ns.load();
+    k.expire_roles = g_expire_roles.load();
     if (k.total_tiles <= 0) return VITCOP_OK;
     CUtensorMap ma, mb;
     if (!make_feat_map(&ma, feat, args.B, args.n, args.D, BM) ||
@@ -1379,13 +1428,15 @@ int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const Gr
 }
 
 bool gram_fits_resident(int B, int n) {
-    static int cooperative = -1;                          // the resident kernel needs a cooperative launch
-    if (cooperative < 0) {
-        int dev = 0, v = 0;
-        cooperative = (cudaGetDevice(&dev) == cudaSuccess &&
-                       cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 0;
+    static std::atomic<int> cooperative[kMaxDevices];     // the resident kernel needs a cooperative launch: 1 yes, 2 no
+    const int dev = current_device();
+    int c = cooperative[dev].load(std::memory_order_relaxed);
+    if (c == 0) {
+        int v = 0;
+        c = (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : 2;
+        cooperative[dev].store(c, std::memory_order_relaxed);
     }
-    if (!cooperative) return false;
+    if (c != 1) return false;
     const int ti = (n + BM - 1) / BM;
     const long long units = (long long)B * (ti + resident_extra_units(ti));
     return units > 0 && units <= (long long)kResidentUnits * num_sms();
@@ -1406,6 +1457,8 @@ int launch_gram_resident(const void* feat, const GramArgs& args, const GramTilin
     k.g.row_end = args.n;
     k.extra_units_per_b = resident_extra_units(k.t.TI);
     k.total_tiles = (long long)args.B * (k.t.TI + k.extra_units_per_b);
+    k.wait_ns = g_wait_ns.load();
+    k.expire_roles = g_expire_roles.load();
     if (k.total_tiles <= 0) return VITCOP_OK;
     if (tiling.BN != BM || k.total_tiles > (long long)kResidentUnits * num_sms()) return VITCOP_ERR_INVALID_ARG;
     CUtensorMap ma, mb;

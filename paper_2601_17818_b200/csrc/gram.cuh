@@ -35,6 +35,11 @@ inline GramTiling make_gram_tiling(int n, int BN) {
     return t;
 }
 
+// Bounded device waits of the Gram kernels: the time after which a wait gives up (0 = the default of 2 s) and, for
+// failure-handling tests, the roles whose waits give up at once (1 load warp, 2 MMA warp, 4 epilogue warps).
+// Applies to launches made after the call.
+void gram_set_wait_debug(unsigned long long limit_ns, int expire_roles);
+
 // Tile width the sweeps use for a problem: wide tiles halve the operand traffic per flop, narrow tiles fill
 // the SMs when the problem is small.
 int gram_pick_bn(int B, int n);

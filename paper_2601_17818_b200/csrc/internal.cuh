@@ -34,7 +34,8 @@ inline bool pdl_allowed(bool requested) { return requested && !kernel_timing_on(
 // ---- launchers (enqueue on `stream`, return VITCOP_OK or VITCOP_ERR_CUDA) -------------------------
 int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
                  int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
-                 cudaStream_t stream, bool late_wait = false);
+                 cudaStream_t stream, bool late_wait = false, bool* launched = nullptr);
+// (`launched`, when given, tells whether a kernel was enqueued at all: an empty span needs none.)
 
 // K-norm to be enqueued in the middle of the filter's kernel chain (vitcop_collaborative_step): it does not depend
 // on the filter, so it runs beside the filter's sweep.
@@ -83,6 +84,26 @@ __device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u &
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Exclusive prefix count of `flag` over a CTA of 1024 threads, in thread order; `total` receives the CTA-wide
+// count.  Must be called by all threads.  warp_sums: shared uint32_t[32].
+__device__ __forceinline__ uint32_t block_prefix_count(bool flag, uint32_t* warp_sums, uint32_t& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t bal = __ballot_sync(0xffffffffu, flag);
+    const uint32_t before = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_sums[warp] = __popc(bal);
+    __syncthreads();
+    uint32_t v = warp_sums[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += t;
+    }
+    total = __shfl_sync(0xffffffffu, v, 31);
+    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
+    __syncthreads();
+    return (warp == 0 ? 0u : base) + before;
 }
 #endif
 

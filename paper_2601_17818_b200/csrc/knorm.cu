@@ -23,7 +23,8 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
     // has completed" meaning "everything before it has completed" for the kernels that follow.
     if (!late_wait) grid_dependency_wait();
     const int b = blockIdx.y;
-    const int nv = vis_len ? vis_len[b] : vis_len_uniform;
+    // a device-side length never reaches past the capacity of the score row (nor, the host has checked, of K)
+    const int nv = max(0, min(vis_len ? vis_len[b] : vis_len_uniform, Nv_cap));
     constexpr int kTok = kKnormThreads / LPR;
     const int sub = threadIdx.x % LPR;
     const int i = blockIdx.x * kTok + threadIdx.x / LPR;
@@ -45,11 +46,13 @@ knorm_kernel(const uint4* __restrict__ K, int H, int d8, int64_t sb, int64_t sh,
 
 int launch_knorm(const void* K, int B, int H, int d, int64_t stride_b, int64_t stride_h, int64_t stride_n,
                  int vis_start, const int32_t* vis_len, int vis_len_uniform, float* score, int Nv_cap,
-                 cudaStream_t stream, bool late_wait) {
+                 cudaStream_t stream, bool late_wait, bool* launched) {
+    if (launched) *launched = false;
     if (B <= 0 || Nv_cap <= 0 || H <= 0) return VITCOP_OK;
     const int d8 = d / 8;
     const int span = vis_len ? Nv_cap : vis_len_uniform;
     if (span <= 0) return VITCOP_OK;
+    if (launched) *launched = true;
     const uint4* Kp = static_cast<const uint4*>(K);
     const int64_t sb = stride_b / 8, sh = stride_h / 8, sn = stride_n / 8;
     int rc = VITCOP_OK;

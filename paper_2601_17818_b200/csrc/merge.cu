@@ -21,25 +21,6 @@ namespace {
 constexpr int kPlanThreads = 1024;
 constexpr int kRowsThreads = 256;
 
-// Exclusive prefix count of `flag` over the CTA in thread order; `total` receives the CTA-wide count.
-__device__ __forceinline__ uint32_t plan_prefix_count(bool flag, uint32_t* warp_sums, uint32_t& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bal = __ballot_sync(0xffffffffu, flag);
-    const uint32_t before = __popc(bal & ((1u << lane) - 1u));
-    if (lane == 0) warp_sums[warp] = __popc(bal);
-    __syncthreads();
-    uint32_t v = warp_sums[lane];
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
-    }
-    total = __shfl_sync(0xffffffffu, v, 31);
-    const uint32_t base = warp == 0 ? 0u : __shfl_sync(0xffffffffu, v, warp - 1);
-    __syncthreads();
-    return base + before;
-}
-
 // Loads the keys (label << 32 | index) of the non-elite tokens, ~0 for everything else, and sorts them.
 template <int E>
 __device__ void sort_members(const int32_t* __restrict__ label, const uint8_t* __restrict__ keep_mask, int n, int T,
@@ -94,8 +75,8 @@ merge_plan_kernel(const int32_t* __restrict__ label, const uint8_t* __restrict__
         const bool tail = valid && (p + 1 >= n || comp[p + 1] == ~0ull || (uint32_t)(comp[p + 1] >> 32) != lab);
         if (valid) members[p] = (uint16_t)(c & 0xFFFFull);
         uint32_t th, tt;
-        const uint32_t hs = heads + plan_prefix_count(head, warp_sums, th);
-        const uint32_t ts = tails + plan_prefix_count(tail, warp_sums, tt);
+        const uint32_t hs = heads + block_prefix_count(head, warp_sums, th);
+        const uint32_t ts = tails + block_prefix_count(tail, warp_sums, tt);
         if (head && hs < (uint32_t)Mcap) {
             merged_label[hs] = (int32_t)lab;
             starts[hs] = p;

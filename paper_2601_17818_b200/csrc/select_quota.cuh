@@ -8,7 +8,7 @@
 namespace vitcop {
 
 constexpr int kSelThreads = 1024;
-constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelWarps = kSelThreads / 32;   // block_prefix_count (internal.cuh) is written for this size
 
 // Ascending key order == the selection order: smaller scores first (or larger, when `largest`),
 // -0 == +0, NaN after everything.
@@ -18,26 +18,6 @@ __device__ __forceinline__ uint32_t order_key(float s, int largest) {
     if (u == 0x80000000u) u = 0u;
     const uint32_t asc = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
     return largest ? ~asc : asc;
-}
-
-// Exclusive prefix count of `flag` over the CTA in thread order; `total` receives the CTA-wide count.
-// Must be called by all threads.  warp_sums: shared uint32_t[kSelWarps].
-__device__ __forceinline__ uint32_t block_prefix_count(bool flag, uint32_t* warp_sums, uint32_t& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bal = __ballot_sync(0xffffffffu, flag);
-    const uint32_t before = __popc(bal & ((1u << lane) - 1u));
-    if (lane == 0) warp_sums[warp] = __popc(bal);
-    __syncthreads();
-    uint32_t v = warp_sums[lane];
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
-    }
-    total = __shfl_sync(0xffffffffu, v, 31);
-    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
-    __syncthreads();
-    return (warp == 0 ? 0u : base) + before;
 }
 
 // Writes keep flags (already decided per element) out in ascending index order.

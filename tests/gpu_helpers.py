@@ -136,20 +136,44 @@ def gpu_similarity_rows(feat_bits, metric, r0, r1):
     return out.cpu().numpy()
 
 
-def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta2, g_parent, g_label, report=None):
-    """Three-level comparison of one sample of the filter against the oracle (see DESIGN notes).
+# Largest share of a sample's tokens whose label may go uncompared with the oracle's (tokens whose parent chain or
+# root legitimately differs because a decision on the way lies inside the tolerance band).  Measured shares are far
+# below this; a widened band or a skipped comparison fails here instead of passing silently.
+MAX_UNCOMPARED_SHARE = 0.03
+
+_VIC_CACHE = {}
+
+
+def oracle_vic_cached(feat_bits, pos, metric, d_c, tau, n_centers, tols):
+    """oracle.vic with a one-entry memo per input (several tests check the same sample of a workload)."""
+    import hashlib
+    h = hashlib.sha1(np.ascontiguousarray(feat_bits).view(np.uint8)).hexdigest()
+    key = (h, None if pos is None else hashlib.sha1(np.ascontiguousarray(pos).view(np.uint8)).hexdigest(),
+           metric, d_c, tau, n_centers, tuple(sorted(tols.items())))
+    if key not in _VIC_CACHE:
+        if feat_bits.shape[0] > 4096:
+            _VIC_CACHE.clear()                 # an n x n fp64 matrix of a long sample is gigabytes: keep one
+        _VIC_CACHE[key] = oracle.vic(feat_bits, pos, metric, d_c, tau, n_centers, tols=tols)
+    return _VIC_CACHE[key]
+
+
+def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta2, g_parent, g_label, report=None,
+                     max_uncompared=MAX_UNCOMPARED_SHARE):
+    """Three-level comparison of one sample of the filter against the oracle.
 
     1. continuous: rho, delta^2 within tolerance;
-    2. discrete vs the oracle: parents / centres / labels equal wherever no decision on the token's path
-       lies inside the tolerance band ("fragile" tokens are excluded and counted);
+    2. discrete vs the oracle: parents equal wherever no decision lies inside the tolerance band; the centre set is
+       one that ranking by the oracle's gamma allows when every gamma moves inside its tolerance interval; labels
+       equal on every token whose actual parent chain and root agree with the oracle's -- the share of tokens left
+       out of that comparison is bounded by `max_uncompared`;
     3. self-consistency, no band: the oracle's discrete steps re-run on the GPU's own fp32 rho / delta^2 /
        parent must reproduce the GPU's parents (up to exact-tie fragility), centres and labels.
     """
     n = feat_bits.shape[0]
     tol = vic_tolerances(metric, d_c, feat_bits)
     RHO_RTOL, D2_ATOL = tol["rho_rtol"], tol["d2_atol"]
-    o = oracle.vic(feat_bits, pos, metric, d_c, tau, n_centers,
-                   tols=dict(tol_rho=RHO_RTOL, tol_d2_abs=D2_ATOL, tol_d2_rel=D2_RTOL, tol_sp=1e-6))
+    o = oracle_vic_cached(feat_bits, pos, metric, d_c, tau, n_centers,
+                          dict(tol_rho=RHO_RTOL, tol_d2_abs=D2_ATOL, tol_d2_rel=D2_RTOL, tol_sp=1e-6))
     # ---- level 1
     assert np.all(rel_err(g_rho, o["rho"]) <= RHO_RTOL), f"rho rel err {rel_err(g_rho, o['rho']).max():.3g}"
     frag = o["fragile"].astype(bool)
@@ -192,24 +216,72 @@ def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta
         assert abs(o["d2"][r, g_label[r]] - dd.min()) <= D2_ATOL + D2_RTOL * dd.min(), "orphan fallback inconsistent"
     assert set(np.unique(g_label).tolist()) <= set(np.flatnonzero(g_isc).tolist())
     # ---- level 2: against the oracle's own discrete results
-    o_isc = o["is_center"].astype(bool)
-    centres_equal = np.array_equal(o_isc, g_isc)
-    n_frag_label = n
-    if centres_equal:
-        # a token is label-robust when every token on its parent chain (up to its root) is parent-robust
-        robust = ~frag
-        chain_ok = robust.copy()
-        order = np.argsort(-o["rho"], kind="stable")
-        for i in order:                       # parents precede children in this order
-            p = o["parent"][i]
-            if not o_isc[i] and p >= 0:
-                chain_ok[i] = robust[i] and chain_ok[p]
-        cmp = chain_ok & ~((o["parent"] < 0) & ~o_isc)
-        assert np.array_equal(g_label[cmp], o["label"][cmp]), "robust labels differ from the oracle"
-        n_frag_label = int((~cmp).sum())
+    o_isc, o_par, o_lab = o["is_center"].astype(bool), o["parent"], o["label"]
+    o_rho, o_d2 = o["rho"], o["delta2"]
+    # 2a. centres.  A token whose parent differs (it is fragile, checked above) may have a different delta, so its
+    #     gamma is free; every other token's gamma lies in [lo, hi] around the oracle's.  The GPU's centre set must
+    #     be a possible top-n_centers of such values: no centre may be certainly below a non-centre.  Orphans
+    #     (gamma = +inf) precede everything and rank among themselves by rho.
+    moved = ~same_parent
+    orphan = o_par < 0
+    e2 = D2_ATOL + D2_RTOL * np.where(orphan, 0.0, o_d2)
+    with np.errstate(invalid="ignore"):
+        hi = o_rho * (1 + RHO_RTOL) * np.sqrt(np.where(orphan, 0.0, o_d2) + e2) * (1 + 1e-6)
+        lo = o_rho * (1 - RHO_RTOL) * np.sqrt(np.maximum(np.where(orphan, 0.0, o_d2) - e2, 0.0)) * (1 - 1e-6)
+    co, cn = g_isc & orphan & ~moved, g_isc & ~orphan & ~moved
+    xo, xn = ~g_isc & orphan & ~moved, ~g_isc & ~orphan & ~moved
+    if xo.any():
+        assert not cn.any(), "a token with a parent is a centre although an orphan is not"
+        if co.any():
+            assert (o_rho[co] * (1 + RHO_RTOL)).min() >= (o_rho[xo] * (1 - RHO_RTOL)).max(), "orphan centres out of order"
+    if cn.any() and xn.any():
+        assert hi[cn].min() >= lo[xn].max(), "centre set impossible under the oracle's gamma within tolerance"
+    # 2b. labels.  Token i is comparable when the GPU took the same path as the oracle: same centre status, same
+    #     parent, and a comparable parent (visited in descending density, so parents come first).  A surplus orphan
+    #     is comparable when the nearest of the GPU's centres is the oracle's choice by a margin beyond tolerance.
+    agree = np.zeros(n, dtype=bool)
+    for i in np.lexsort((np.arange(n), -o_rho)):
+        if o_isc[i] or g_isc[i]:
+            agree[i] = o_isc[i] and g_isc[i]
+        elif o_par[i] < 0:
+            if g_parent[i] < 0 and len(cs) > 0:
+                dd = o["d2"][i, cs]
+                k = int(np.argmin(dd))
+                rest = np.delete(dd, k)
+                clear = len(rest) == 0 or rest.min() - dd[k] > 2 * (D2_ATOL + D2_RTOL * dd[k])
+                agree[i] = clear and cs[k] == o_lab[i]
+        else:
+            agree[i] = same_parent[i] and agree[o_par[i]]
+    assert np.array_equal(g_label[agree], o_lab[agree]), "labels differ from the oracle on an identical path"
+    uncompared = int(n - agree.sum())
+    stats = dict(n=n, fragile_parent=int(frag.sum()), parent_mismatch=int(moved.sum()),
+                 centre_diff=int((o_isc != g_isc).sum()), label_uncompared=uncompared,
+                 label_mismatch=int((g_label != o_lab).sum()), rho_err=float(rel_err(g_rho, o_rho).max()))
     if report is not None:
-        report.append(dict(n=n, fragile_parent=int(frag.sum()), parent_mismatch=int((~same_parent).sum()),
-                           centres_equal=bool(centres_equal), label_uncompared=n_frag_label,
-                           label_mismatch=int((g_label != o["label"]).sum()),
-                           rho_err=float(rel_err(g_rho, o["rho"]).max())))
+        report.append(stats)
+    assert uncompared <= max_uncompared * n + 2, f"too many labels left uncompared: {stats}"
     return o
+
+
+def oracle_quota_band_check(score64, label, gpu_keep, budget, rtol):
+    """Kept-set comparison of the cluster-quota selection (Eq. 5) of one sequence with the tolerance band at each
+    cluster's cut: cluster c keeps exactly its quota q_c; inside a cluster, tokens whose oracle score lies within
+    `rtol` (relative) of the scores on either side of the cut may swap; every other token must agree.
+    Returns the number of differing tokens."""
+    want, nc, quota = oracle.select_quota(score64, label, budget)
+    assert want is not None and len(gpu_keep) == len(want)
+    assert np.all(np.diff(gpu_keep) > 0)
+    diff = np.setxor1d(gpu_keep, want)
+    kept = np.zeros(len(score64), dtype=bool)
+    kept[gpu_keep] = True
+    for c in np.unique(label[diff]) if len(diff) else []:
+        members = np.flatnonzero(label == c)
+        q = int(quota[c])
+        assert int(kept[members].sum()) == q, "a cluster's kept count differs from its quota"
+        srt = np.sort(score64[members])
+        assert 0 < q < len(members)
+        lo, hi = srt[q - 1], srt[q]
+        d = diff[label[diff] == c]
+        assert np.all((score64[d] >= lo - rtol * abs(lo)) & (score64[d] <= hi + rtol * abs(hi))), \
+            f"cluster {c}: tokens outside the tolerance band at the cut differ"
+    return int(len(diff))

@@ -115,11 +115,12 @@ def test_argument_validation_of_the_wider_entry_points(L):
     assert L.vitcop_cls_saliency(fake, odd, 1, 1, 4, 8, 0.5, fake, null, ws, 1 << 20, null) == vb.ERR_UNSUPPORTED
     assert L.vitcop_cls_saliency(fake, fake, 1, 1, 4, 8, 0.5, fake, null, ws, 16, null) == vb.ERR_WORKSPACE
     # one-call Stage II: needs labels out, a valid metric / cutoff, D % 64, a workspace
-    args = lambda feat=fake, D=64, f=fp, lab=fake, wsb=1 << 24: (feat, null, D, C.byref(f), null, a, null, 1, 1, 8, 8, 8, 0, 4, 2, null, b, null, 8, null, fake, lab, fake, null, null, null, ws, wsb, null)
+    args = lambda feat=fake, D=64, f=fp, lab=fake, wsb=1 << 24, B=1: (feat, null, D, C.byref(f), null, a, null, B, 1, 8, 8, 8, 0, 4, 2, null, b, null, 8, null, fake, lab, fake, null, null, null, null, null, null, ws, wsb, null)
     assert L.vitcop_collaborative_step(*args(lab=null)) == vb.ERR_INVALID_ARG
     assert L.vitcop_collaborative_step(*args(f=vb.FilterParams(0, 0.0, 0.6, 0.05, 0))) == vb.ERR_INVALID_ARG
     assert L.vitcop_collaborative_step(*args(D=72)) == vb.ERR_UNSUPPORTED
     assert L.vitcop_collaborative_step(*args(wsb=64)) == vb.ERR_WORKSPACE
+    assert L.vitcop_collaborative_step(*args(B=65536, wsb=1 << 40)) == vb.ERR_UNSUPPORTED      # as its sibling calls
     assert vb.vitcop_workspace_bytes(vb.OP_COLLAB_STEP, B=2, Nv=100, D=64) > vb.vitcop_workspace_bytes(vb.OP_FILTER, B=2, Nv=100, D=64)
     assert vb.vitcop_workspace_bytes(vb.OP_MERGE, B=2, Nv=100, N=10) >= 256 + 2 * 100 * 2
     assert vb.vitcop_workspace_bytes(vb.OP_SALIENCY, B=2, H=4, N=33) >= 2 * 4 * 33 * 4

@@ -77,3 +77,60 @@ def test_filter_full_c4():
     ok = par >= 0
     rho = g.rho[0]
     assert np.all((rho[par[ok]] > rho[ok]) | ((rho[par[ok]] == rho[ok]) & (par[ok] < np.flatnonzero(ok))))
+
+
+# Stage II through the one call the benchmark times, compared DIRECTLY with the oracle: K-norm scores (computed in
+# part by the side warps of the one-kernel sweep on c0/c1, by the stand-alone kernel elsewhere), the clustering by
+# the three-level rule, the quota selection and the compacted rows.
+@pytest.mark.parametrize("name,samples", [("tiny", None), ("c0", None), ("c1", None), ("c2", (7,)), ("c3", (3,)),
+                                          ("c4", (1,))])
+def test_collaborative_step_vs_oracle(name, samples):
+    from gpu_helpers import DEV, oracle_quota_band_check
+    w = W.workload(name)
+    B, n = w.B, w.Nv
+    f, p = W.make_features(w), W.make_positions(w)
+    K_b, V_b = W.make_kv(w, 0, n)
+    hid_b = W.make_hidden(w)
+    budget = w.budgets[0]
+    Ncap = w.T + budget
+    z = lambda *s, dt: torch.zeros(s, dtype=dt, device=DEV)
+    ho, Ko, Vo = (z(B, Ncap, w.Dh, dt=torch.bfloat16), z(B, w.H, Ncap, w.d, dt=torch.bfloat16),
+                  z(B, w.H, Ncap, w.d, dt=torch.bfloat16))
+    olen, kpos = z(B, dt=torch.int32), z(B, Ncap, dt=torch.int32)
+    label, ncl = z(B, n, dt=torch.int32), z(B, dt=torch.int32)
+    rho, d2, par = z(B, n, dt=torch.float32), z(B, n, dt=torch.float32), z(B, n, dt=torch.int32)
+    score, kidx, nkeep = z(B, n, dt=torch.float32), z(B, n, dt=torch.int32), z(B, dt=torch.int32)
+    ws = vb.alloc_workspace(vb.OP_COLLAB_STEP, B=B, Nv=n, D=w.D)
+    vb.vitcop_collaborative_step(vb.bf16_tensor(f), torch.from_numpy(p.copy()).to(DEV), vb.bf16_tensor(hid_b),
+                                 vb.bf16_tensor(K_b), vb.bf16_tensor(V_b), w.vis_start, budget, ho, Ko, Vo, olen, label,
+                                 ncl, ws, metric=0, d_c=w.d_c, tau=w.tau, n_centers=w.n_centers, kept_pos=kpos,
+                                 score_out=score, keep_idx_out=kidx, n_keep_out=nkeep, rho=rho, delta2=d2, parent=par)
+    assert vb.vitcop_poll_status(ws) == vb.OK
+    g_score, g_idx, g_nk = score.cpu().numpy(), kidx.cpu().numpy(), nkeep.cpu().numpy()
+    g_label, g_rho, g_d2, g_par = label.cpu().numpy(), rho.cpu().numpy(), d2.cpu().numpy(), par.cpu().numpy()
+    g_ho, g_Ko, g_Vo = vb.bf16_bits(ho), vb.bf16_bits(Ko), vb.bf16_bits(Vo)
+    g_olen, g_pos = olen.cpu().numpy(), kpos.cpu().numpy()
+    assert np.all(ncl.cpu().numpy() == w.n_centers)
+    # Eq. 4
+    o_score = oracle.knorm(K_b, w.vis_start, n)
+    assert np.all(rel_err(g_score, o_score) <= KNORM_RTOL)
+    # Algorithm 2
+    rep = []
+    for b in (range(B) if samples is None else samples):
+        check_vic_sample(f[b], p[b], 0, w.d_c, w.tau, w.n_centers, g_rho[b], g_d2[b], g_par[b], g_label[b], rep)
+    print("collaborative step", name, rep)
+    diffs = 0
+    for b in range(B):
+        keep = g_idx[b, : g_nk[b]]
+        # Eq. 5 / Algorithm 3: exact on the kernel's own fp32 scores; vs the oracle's scores up to the band at each cut
+        want, nc, _ = oracle.select_quota(g_score[b].astype(np.float64), g_label[b], budget)
+        assert nc == w.n_centers and np.array_equal(keep, want)
+        diffs += oracle_quota_band_check(o_score[b], g_label[b], keep, budget, KNORM_RTOL)
+        # compaction: bit-exact rows
+        o = oracle.compact(hid_b[b], K_b[b], V_b[b], w.N, w.vis_start, n, keep, Ncap)
+        L = o["out_len"]
+        assert g_olen[b] == L == w.T + g_nk[b]
+        assert np.array_equal(g_pos[b, :L], o["kept_pos"][:L])
+        assert np.array_equal(g_ho[b, :L], o["hidden"][:L])
+        assert np.array_equal(g_Ko[b, :, :L], o["K"][:, :L]) and np.array_equal(g_Vo[b, :, :L], o["V"][:, :L])
+    print("collaborative step", name, "selection differences inside the band:", diffs)

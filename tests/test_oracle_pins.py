@@ -359,6 +359,111 @@ def test_spatial_mask_hand_example():
     assert oracle.vic_parents(d2, pos, rho, 0.4999)[1][0] == -1
 
 
+# The robustness report of oracle.vic_parents decides which tokens a lower-precision implementation may
+# legitimately disagree on, so its band must be neither too narrow nor too wide.  Hand-built cases: the answer is
+# known by construction on each side of every tolerance.
+def _frag(d2, pos, rho, tau, **tols):
+    _, parent, frag = oracle.vic_parents(np.asarray(d2, dtype=np.float64), pos, np.asarray(rho, dtype=np.float64),
+                                         tau, want_fragile=True, **tols)
+    return parent.tolist(), frag.astype(bool).tolist()
+
+
+def _sym(n, entries, fill=9.0):
+    d2 = np.full((n, n), fill)
+    np.fill_diagonal(d2, 0.0)
+    for (i, j), v in entries.items():
+        d2[i, j] = d2[j, i] = v
+    return d2
+
+
+@pytest.mark.parametrize("factor,expect", [(0.5, True), (2.0, False)])
+def test_fragile_report_distance_band(factor, expect):
+    # token 0 has two denser candidates: 1 at d2 = 1 (the parent) and 2 at d2 = 1 + factor * band, where
+    # band = tol_abs + tol_rel * 1: half a band away the runner-up could win, two bands away it could not
+    tol_abs, tol_rel = 3e-6, 1e-5
+    band = tol_abs + tol_rel * 1.0
+    d2 = _sym(3, {(0, 1): 1.0, (0, 2): 1.0 + factor * band, (1, 2): 4.0})
+    parent, frag = _frag(d2, None, [1.0, 2.0, 3.0], -1.0, tol_d2_abs=tol_abs, tol_d2_rel=tol_rel)
+    assert parent == [1, 2, -1]
+    assert frag == [expect, False, False]
+    # the absolute and the relative part each count on their own
+    for kw in (dict(tol_d2_abs=band), dict(tol_d2_rel=band)):
+        assert _frag(d2, None, [1.0, 2.0, 3.0], -1.0, **kw)[1][0] is expect
+
+
+@pytest.mark.parametrize("factor,expect", [(0.5, True), (2.0, False)])
+def test_fragile_report_density_band(factor, expect):
+    tol = 1e-4
+    # (a) a closer token whose density lies just BELOW token 0's: not a candidate, but it could become one
+    rho = [1.0, 2.0, 1.0 - factor * tol]
+    d2 = _sym(3, {(0, 1): 1.0, (0, 2): 0.25, (1, 2): 4.0})
+    parent, frag = _frag(d2, None, rho, -1.0, tol_rho=tol)
+    assert parent[0] == 1 and frag[0] is expect
+    # (b) the parent's own density lies just ABOVE token 0's: it could stop being a candidate
+    rho = [1.0, 1.0 + factor * tol, 0.5]
+    parent, frag = _frag(_sym(3, {(0, 1): 1.0, (0, 2): 0.25, (1, 2): 4.0}), None, rho, -1.0, tol_rho=tol)
+    assert parent[0] == 1 and frag[0] is expect
+    # (c) an orphan (densest token) with a near-equal neighbour could gain a parent
+    rho = [1.0, 1.0 - factor * tol, 0.5]
+    parent, frag = _frag(_sym(3, {(0, 1): 1.0}), None, rho, -1.0, tol_rho=tol)
+    assert parent[0] == -1 and frag[0] is expect
+    # a farther token cannot matter however close its density is
+    rho = [1.0, 2.0, 1.0 - 0.5 * tol]
+    assert _frag(_sym(3, {(0, 1): 1.0, (0, 2): 1.5, (1, 2): 4.0}), None, rho, -1.0, tol_rho=tol)[1][0] is False
+
+
+@pytest.mark.parametrize("factor,expect", [(0.5, True), (2.0, False)])
+def test_fragile_report_spatial_band(factor, expect):
+    tau, tol = 0.5, 1e-3                                   # positions on the x axis: distances exact in fp32 -> fp64
+    x = lambda v: np.array([[0.0, 0.0], [np.float32(v), 0.0], [0.25, 0.0]], dtype=np.float32)
+    rho = [1.0, 2.0, 3.0]
+    # (a) a closer, denser token just OUTSIDE the radius: excluded, but it could slip inside
+    d2 = _sym(3, {(0, 1): 0.25, (0, 2): 1.0, (1, 2): 4.0})
+    parent, frag = _frag(d2, x(tau * (1 + factor * tol)), rho, tau, tol_sp=tol)
+    assert parent[0] == 2 and frag[0] is expect
+    # (b) the parent itself just INSIDE the radius: it could slip outside
+    d2 = _sym(3, {(0, 1): 0.25, (0, 2): 1.0, (1, 2): 4.0})
+    parent, frag = _frag(d2, x(tau * (1 - factor * tol)), rho, tau, tol_sp=tol)
+    assert parent[0] == 1 and frag[0] is expect
+
+
+def test_fragile_report_without_tolerances_flags_exact_ties_only():
+    rng = np.random.default_rng(5)
+    n = 80
+    a = rng.random((n, n)) + 0.1
+    d2 = (a + a.T) / 2
+    np.fill_diagonal(d2, 0.0)
+    rho = rng.random(n) + 1.0
+    pos = rng.random((n, 2)).astype(np.float32)
+    for kw in (dict(pos=None, tau=-1.0), dict(pos=pos, tau=0.45)):
+        parent, frag = _frag(d2, kw["pos"], rho, kw["tau"])
+        assert not any(frag)                               # continuous random values: no ties, nothing fragile
+    # plant (1) an exact tie in distance between the parent of token t and another denser token, and
+    #       (2) an exact tie in density between a token u and a closer token
+    parent, _ = _frag(d2, None, rho, -1.0)
+    order = np.argsort(rho)
+    t = int(order[10])                                     # a token with many denser ones
+    denser = [int(j) for j in order[11:] if j != parent[t]]
+    other = denser[0]
+    d2b = d2.copy()
+    for j in (other, parent[t]):                           # both at the same distance, closer than everything else
+        d2b[t, j] = d2b[j, t] = 2e-3
+    u = int(order[30])
+    v = int(order[5])                                      # strictly less dense than u ...
+    rho_b = rho.copy()
+    rho_b[v] = rho_b[u]                                    # ... now exactly as dense
+    d2b[u, v] = d2b[v, u] = 1e-3                           # and closer than anything else
+    parent_b, frag_b = _frag(d2b, None, rho_b, -1.0)
+    flagged = set(np.flatnonzero(frag_b).tolist())
+    assert t in flagged and u in flagged and v in flagged
+    # every flagged token owes it to one of the two planted ties
+    for i in flagged:
+        best = d2b[i, parent_b[i]] if parent_b[i] >= 0 else np.inf
+        ties_d = [j for j in range(n) if j not in (i, parent_b[i]) and rho_b[j] >= rho_b[i] and d2b[i, j] == best]
+        ties_r = [j for j in range(n) if j != i and rho_b[j] == rho_b[i] and d2b[i, j] <= best]
+        assert ties_d or ties_r, i
+
+
 def test_all_orphans_fall_back_to_nearest_centre():
     w = W.workload("tiny")
     f = W.make_features(w)[0][:60]

@@ -29,7 +29,11 @@ def _outputs(B, H, Ncap, d, Dh, n):
                 score=z(B, n, dt=torch.float32), kidx=z(B, n, dt=torch.int32), nkeep=z(B, dt=torch.int32))
 
 
-def _both(w, step, n_vis, budget, label):
+def _both(w, step, n_vis, budget, label, own_buffers):
+    """One problem through vitcop_prune_step (ordinary workspace) and through vitcop_prune_step_static.
+
+    own_buffers=False leaves score / keep list / counts to the call: the static variant then keeps them in its
+    built-in scratch, which is the memory this test is about."""
     K, V = W.make_kv(w, step, n_vis)
     hid = W.make_hidden(w)[:, : w.T + n_vis]
     tK, tV, th = vb.bf16_tensor(K), vb.bf16_tensor(V), vb.bf16_tensor(np.ascontiguousarray(hid))
@@ -42,27 +46,52 @@ def _both(w, step, n_vis, budget, label):
                          n_keep_out=ref["nkeep"])
     assert vb.vitcop_poll_status(ws) == vb.OK
     got = _outputs(w.B, w.H, Ncap, w.d, w.Dh, n_vis)
-    vb.vitcop_prune_step_static(th, tK, tV, w.vis_start, n_vis, n_vis, budget, got["ho"], got["Ko"], got["Vo"],
-                                got["olen"], label=lab, kept_pos=got["kpos"], score_out=got["score"],
-                                keep_idx_out=got["kidx"], n_keep_out=got["nkeep"])
+    own = dict(score_out=got["score"], keep_idx_out=got["kidx"], n_keep_out=got["nkeep"]) if own_buffers else {}
     torch.cuda.synchronize()
-    r_score, g_score = ref["score"].cpu().numpy(), got["score"].cpu().numpy()
-    assert np.all(np.abs(g_score - r_score) <= KNORM_RTOL * np.abs(r_score))
+    held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+    vb.vitcop_prune_step_static(th, tK, tV, w.vis_start, n_vis, n_vis, budget, got["ho"], got["Ko"], got["Vo"],
+                                got["olen"], label=lab, kept_pos=got["kpos"], **own)
+    torch.cuda.synchronize()
+    grown = (torch.cuda.memory_allocated() - held, free - torch.cuda.mem_get_info()[0])
     nk = ref["nkeep"].cpu().numpy()
-    assert np.array_equal(got["nkeep"].cpu().numpy(), nk) and nk.max() > 0
+    assert nk.max() > 0
     assert np.array_equal(got["olen"].cpu().numpy(), ref["olen"].cpu().numpy())
-    for b in range(w.B):
-        assert np.array_equal(got["kidx"].cpu().numpy()[b, : nk[b]], ref["kidx"].cpu().numpy()[b, : nk[b]])
+    assert np.array_equal(ref["olen"].cpu().numpy(), w.T + nk)
+    if own_buffers:
+        r_score, g_score = ref["score"].cpu().numpy(), got["score"].cpu().numpy()
+        assert np.all(np.abs(g_score - r_score) <= KNORM_RTOL * np.abs(r_score))
+        assert np.array_equal(got["nkeep"].cpu().numpy(), nk)
+        for b in range(w.B):
+            assert np.array_equal(got["kidx"].cpu().numpy()[b, : nk[b]], ref["kidx"].cpu().numpy()[b, : nk[b]])
     assert torch.equal(got["kpos"], ref["kpos"])
     for name in ("ho", "Ko", "Vo"):
         assert torch.equal(got[name].view(torch.int16), ref[name].view(torch.int16)), name
+    return grown
 
 
 def test_prune_step_static_matches_prune_step_twice_in_a_row():
     w = W.workload("tiny")
     labels = W.make_labels(5, w.B, w.Nv, w.n_centers)
-    _both(w, 0, w.Nv, w.budgets[0], labels)         # first call: quota mode, full span
-    _both(w, 1, 77, 13, None)                       # second call: plain mode, other sizes, stale scratch underneath
+    _both(w, 0, w.Nv, w.budgets[0], labels, own_buffers=True)    # first call: quota mode, full span
+    # second call: plain mode, other (smaller) sizes, scores / keep list / counts in the built-in scratch, which
+    # still holds what the larger first call left there
+    _both(w, 1, 77, 13, None, own_buffers=False)
+    # third: quota mode again on the scratch, over the plain call's leftovers
+    grown = _both(w, 2, w.Nv, w.budgets[1], labels, own_buffers=False)
+    # the call itself obtains no device memory, neither from torch's allocator nor from the driver (looked at
+    # around the third call: every kernel it launches had been loaded by then)
+    assert grown == (0, 0)
+
+
+def test_prune_step_static_uses_the_whole_scratch_near_its_limit():
+    """B * Nv_cap just below the limit: the keep list and the counts sit at the far end of the 4 MiB array."""
+    import dataclasses
+    w = dataclasses.replace(W.workload("tiny"), B=32, Nv=16256, T=8, H=1, d=8, Dh=8, budgets=(300, 100))
+    need = vb.vitcop_workspace_bytes(vb.OP_PRUNE_STEP, B=w.B, Nv=w.Nv)
+    assert (4 << 20) - 64 * 1024 < need <= (4 << 20)
+    _both(w, 0, w.Nv, 300, None, own_buffers=False)
+    labels = W.make_labels(9, w.B, w.Nv, 40)
+    _both(w, 1, w.Nv, 500, labels, own_buffers=False)
 
 
 def test_prune_step_static_refuses_oversized_problems():
