@@ -35,3 +35,19 @@ def whole_job_rate(units_per_rank_per_step: float, steps: int, total_ms_this_ran
     scaling: per-GPU work is fixed) in the time of the slowest rank."""
     ms = max_over_ranks(total_ms_this_rank, device)
     return world() * units_per_rank_per_step * steps / (ms * 1e-3)
+
+
+def launch_ranks(n: int, argv, env=None) -> int:
+    """Starts `n` ranks of `argv` (a script path followed by its arguments) on this node, one per GPU, under
+    torch.distributed.run with a loopback rendezvous on a free port, and returns the launcher's exit code.  This is
+    what `bench.py --gpus N` does when it is invoked without a torchrun environment."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(n)}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), *argv]
+    return subprocess.call(cmd, env=dict(os.environ if env is None else env))

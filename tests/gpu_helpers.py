@@ -236,22 +236,33 @@ def check_vic_sample(feat_bits, pos, metric, d_c, tau, n_centers, g_rho, g_delta
             assert (o_rho[co] * (1 + RHO_RTOL)).min() >= (o_rho[xo] * (1 - RHO_RTOL)).max(), "orphan centres out of order"
     if cn.any() and xn.any():
         assert hi[cn].min() >= lo[xn].max(), "centre set impossible under the oracle's gamma within tolerance"
-    # 2b. labels.  Token i is comparable when the GPU took the same path as the oracle: same centre status, same
-    #     parent, and a comparable parent (visited in descending density, so parents come first).  A surplus orphan
-    #     is comparable when the nearest of the GPU's centres is the oracle's choice by a margin beyond tolerance.
-    agree = np.zeros(n, dtype=bool)
-    for i in np.lexsort((np.arange(n), -o_rho)):
-        if o_isc[i] or g_isc[i]:
-            agree[i] = o_isc[i] and g_isc[i]
-        elif o_par[i] < 0:
-            if g_parent[i] < 0 and len(cs) > 0:
-                dd = o["d2"][i, cs]
-                k = int(np.argmin(dd))
-                rest = np.delete(dd, k)
-                clear = len(rest) == 0 or rest.min() - dd[k] > 2 * (D2_ATOL + D2_RTOL * dd[k])
-                agree[i] = clear and cs[k] == o_lab[i]
-        else:
-            agree[i] = same_parent[i] and agree[o_par[i]]
+    # 2b. labels.  Token i is comparable when the path the GPU took must end in the oracle's label: a centre of both;
+    #     or a token whose GPU parent p is comparable and lies in the oracle's cluster of i (p is the oracle's own
+    #     parent, or -- for a fragile token -- another member of the same cluster); or a surplus orphan for which the
+    #     nearest of the GPU's centres is the oracle's choice by a margin beyond tolerance.
+    state = np.zeros(n, dtype=np.int8)                     # 0 unknown, 1 comparable, 2 not
+    for i0 in range(n):
+        path, i = [], i0
+        while state[i] == 0 and len(path) <= n:
+            if o_isc[i] or g_isc[i]:
+                state[i] = 1 if (o_isc[i] and g_isc[i]) else 2
+            elif g_parent[i] < 0:
+                state[i] = 2
+                if o_par[i] < 0 and len(cs) > 0:
+                    dd = o["d2"][i, cs]
+                    k = int(np.argmin(dd))
+                    rest = np.delete(dd, k)
+                    clear = len(rest) == 0 or rest.min() - dd[k] > 2 * (D2_ATOL + D2_RTOL * dd[k])
+                    if clear and cs[k] == o_lab[i]:
+                        state[i] = 1
+            else:
+                path.append(i)
+                i = int(g_parent[i])
+        ok_up = state[i] == 1
+        for j in reversed(path):
+            ok_up = ok_up and o_lab[g_parent[j]] == o_lab[j]
+            state[j] = 1 if ok_up else 2
+    agree = state == 1
     assert np.array_equal(g_label[agree], o_lab[agree]), "labels differ from the oracle on an identical path"
     uncompared = int(n - agree.sum())
     stats = dict(n=n, fragile_parent=int(frag.sum()), parent_mismatch=int(moved.sum()),

@@ -51,3 +51,39 @@ def test_single_process_is_its_own_job():
     assert replicas.world() == 1
     assert replicas.max_over_ranks(3.5) == 3.5
     assert replicas.whole_job_rate(100, 2, 4.0) == 100 * 2 / 4e-3
+
+
+def test_launcher_starts_the_ranks_itself(tmp_path):
+    """`bench.py --gpus N` invoked plainly re-launches itself through replicas.launch_ranks; here the same launcher
+    starts two CPU ranks of a stub step and rank 0 reports the whole job."""
+    import json
+    import sys
+    here = os.path.dirname(os.path.abspath(__file__))
+    out = tmp_path / "line.json"
+    env = dict(os.environ, PYTHONPATH=os.pathsep.join([os.path.dirname(here)] + sys.path))
+    rc = replicas.launch_ranks(2, [os.path.join(here, "replica_stub.py"), "--gpus", "2", "--steps", "3", "--out", str(out)],
+                               env=env)
+    assert rc == 0
+    line = json.loads(out.read_text())
+    assert line["n_gpus"] == 2 and line["gpus_arg"] == 2
+    assert line["ms"] >= 3 * 0.01 * 2 * 1e3 * 0.9            # the slower rank's time
+    assert abs(line["value"] - 2 * 1000 * 3 / (line["ms"] * 1e-3)) / line["value"] < 0.35
+
+
+def test_bench_relaunches_itself_when_asked_for_several_gpus(monkeypatch):
+    import importlib.util
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    seen = {}
+    monkeypatch.setattr(replicas, "launch_ranks", lambda n, argv, env=None: seen.update(n=n, argv=argv) or 0)
+    monkeypatch.delenv("RANK", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "7"])
+    try:
+        bench.main()
+    except SystemExit as e:
+        assert e.code == 0
+    assert seen["n"] == 4 and seen["argv"][1:] == ["--gpus", "4", "--steps", "7"]
+    assert seen["argv"][0].endswith("bench.py")
