@@ -631,6 +631,15 @@ def run_ours(args):
 
     w = W.workload(args.workload)
     solo = rank == 0 and world == 1
+    if args.profile_run:
+        # for a profiler: the schedule of one workload, warm-up + steps, nothing else launched by this library
+        b = Bench(w, torch, vb, dev, flush, peaks, replicas)
+        for _ in range(args.warmup + args.steps):
+            flush.zero_()
+            b.sc.run()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": w.name, "steps": args.steps, "warmup": args.warmup}))
+        return
     head = Bench(w, torch, vb, dev, flush, peaks, replicas).run(
         args.steps, args.warmup, max(5, min(args.steps, 20)),
         args.cpu_seconds if solo and not args.no_cpu_baseline else 0, True, local)
@@ -677,6 +686,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true", help="measure the headline workload only")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="length of the CPU-oracle timing leg")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="only run the workload's schedule (warm-up + steps) and exit: the command a profiler wraps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.gpus > 1 and "RANK" not in os.environ:

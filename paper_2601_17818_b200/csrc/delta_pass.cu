@@ -1,0 +1,290 @@
+// Eq. 3 (Algorithm 2, step 2) from stored Gram tiles: per token the nearest denser token inside the spatial radius.
+//
+// The density sweep (gram.cu, GRAM_RHO) has just computed every Gram value on the tensor cores and written the tiles
+// it visited to the workspace; the densities it produces order the tokens, so Eq. 3 needs a second look at every
+// pair.  Reading a pair back costs 4 bytes; recomputing it costs 2 D flop, several times more of the machine.  This
+// kernel therefore streams the tiles from memory (L2 for the smaller problems, HBM for the long ones) and does the
+// per-pair work of Eq. 3 with plain ALU instructions -- the same arithmetic, in the same order, as the delta epilogue
+// of the one-kernel sweep, so both give the same bits.
+//
+// One CTA of 8 warps per tile, up to four CTAs per SM, a persistent grid; every CTA takes one contiguous run of the
+// tile numbering, i.e. consecutive row blocks against one column block (see below why).  Warp w owns
+// the rows 32 (w % 4) .. + 31 of the tile (one per lane) and the column half w / 4; a thread walks its half eight
+// columns at a time (two 16-byte loads, the next two already in flight), keeps its row's minimum, and the warp reduces
+// each column over its 32 rows with redux / ballot.  The four row quarters of a column and the two halves of a row are
+// combined through shared memory in a fixed order (ties keep the lower index) and folded into the per-token packed
+// minima with one 64-bit atomicMin each.
+//
+// Most pairs cannot matter: a pair serves its row token only if its d^2 does not exceed the best that token has so
+// far, and its column token likewise (and a pair serves only one of the two: the less dense one).  Both bounds are read from the packed minima when the tile starts (other CTAs
+// keep lowering them, a stale bound is merely looser) and tightened as the tile goes.  A thread first computes d^2 of
+// its eight pairs and tests them against the two bounds (with <=: an equal distance at a lower index still wins);
+// one redux.or tells the warp which of the eight columns hold a candidate at all, and only those columns go through
+// the spatial test, the density comparison, the row update and the column reduction.  What is skipped could not
+// have changed any minimum, so the result is the same as without the test.
+// The bounds only bite once a token has seen some of its candidates, so the order of the work matters: a CTA walks
+// down one column block, whose tokens thus meet their candidates one row block after the other (their bounds stay in
+// shared memory from tile to tile), while the CTAs of other column blocks reach any given row block at different
+// times, so that a row token's bound in global memory has been lowered by the time most of them read it.
+#include "gram.cuh"
+
+namespace vitcop {
+namespace {
+
+constexpr int BM = kGramBM;
+constexpr int kDpSlices = 2;                              // column slices of a tile, four warps each
+constexpr int kDpThreads = 128 * kDpSlices;
+constexpr int kDpCtasPerSm = 4;
+constexpr float kInf = __builtin_huge_valf();
+
+// Bits of the largest d^2 that can still improve the packed minimum at `p` (an equal d^2 with a lower index would):
+// the d^2 it holds, or +inf when it holds none.  Read from L2: other CTAs lower it while this one runs.
+__device__ __forceinline__ int bound_of(const unsigned long long* p) {
+    const unsigned long long v = __ldcg(p);
+    return v == ~0ull ? 0x7f800000 : (int)(uint32_t)(v >> 32);
+}
+
+__device__ __forceinline__ float4 ld_tile(const float4* p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <int BN, int METRIC, bool SPATIAL>
+__global__ void __launch_bounds__(kDpThreads, kDpCtasPerSm)
+delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_tiles) {
+    constexpr int NS = kDpSlices;
+    constexpr int kSliceCols = BN / NS;
+    constexpr int kGroups = kSliceCols / 8;
+    __shared__ __align__(16) float colw[BN], cola[BN], colrho[BN], colx[BN], coly[BN];
+    __shared__ __align__(16) int colthr[BN];               // bits of the largest d^2 that can still serve column j
+    __shared__ unsigned long long colbest[BN];             // packed (d^2 bits, row) minimum of every column of the tile
+    __shared__ float rowred[(kDpSlices - 1) * BM];
+    __shared__ int rowidx[(kDpSlices - 1) * BM];
+    __shared__ float roww[BM], rowa[BM], rowrho[BM], rowx[BM], rowy[BM];
+
+    // A kernel queued behind this one that does not depend on it may share the SMs from the start.
+    grid_dependency_launch_dependents();
+    grid_dependency_wait();                                // rho, the factors and the tiles come from the preceding kernels
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int quarter = warp & 3, slice = warp >> 2;
+    const int rl = quarter * 32 + lane;                    // tile-local row of this thread
+
+    const long long t_begin = total_tiles * blockIdx.x / gridDim.x, t_end = total_tiles * (blockIdx.x + 1) / gridDim.x;
+    int prev_b = -1, prev_tj = -1;
+    for (long long t = t_begin; t < t_end; ++t) {
+        int b, ti, tj;
+        decode_sym_tile(tl, t, b, ti, tj);
+        const bool same_cols = b == prev_b && tj == prev_tj;       // the column block of the previous tile: its constants stay
+        prev_b = b;
+        prev_tj = tj;
+        const int I0 = ti * BM, J0 = tj * BN;
+        const int i = I0 + rl;
+        const bool row_valid = i < g.n;
+        const size_t bo = (size_t)b * g.n;
+
+        // the first two loads of this thread's slice travel while the tile's constants are fetched
+        const float4* src = reinterpret_cast<const float4*>(g.gram_tiles + (size_t)t * gram_tile_floats(BN)) +
+                            (size_t)(slice * kSliceCols / 4) * BM + rl;
+        float4 cur0 = ld_tile(src), cur1 = ld_tile(src + BM);
+
+        for (int it = threadIdx.x; it < 2 * BN + 2 * BM; it += kDpThreads) {
+            if (it < BN) {
+                const int j = J0 + it;
+                const bool cv = j < g.n;
+                const int bound = cv ? bound_of(g.best + bo + j) : (int)0x80000000;
+                colbest[it] = ~0ull;
+                if (same_cols) {
+                    colthr[it] = min(colthr[it], bound);
+                } else {
+                    colthr[it] = bound;
+                    colw[it] = cv ? g.w[bo + j] : 0.f;
+                    if (METRIC == 1) cola[it] = cv ? g.a[bo + j] : 0.f;
+                }
+            } else if (it < 2 * BN) {
+                if (same_cols) continue;
+                const int ce = it - BN, j = J0 + ce;
+                float rj = 0.f;
+                float2 pj = make_float2(0.f, 0.f);
+                if (j < g.n) {
+                    if (SPATIAL) pj = *reinterpret_cast<const float2*>(g.pos + 2 * (bo + j));
+                    rj = g.rho[bo + j];
+                }
+                colrho[ce] = rj;
+                if (SPATIAL) { colx[ce] = pj.x; coly[ce] = pj.y; }
+            } else if (it < 2 * BN + BM) {
+                const int r = it - 2 * BN, ir = I0 + r;
+                const bool rv = ir < g.n;
+                roww[r] = rv ? g.w[bo + ir] : 0.f;
+                if (METRIC == 1) rowa[r] = rv ? g.a[bo + ir] : 0.f;
+            } else {
+                const int r = it - 2 * BN - BM, ir = I0 + r;
+                float rr = 0.f;
+                float2 pr = make_float2(0.f, 0.f);
+                if (ir < g.n) {
+                    if (SPATIAL) pr = *reinterpret_cast<const float2*>(g.pos + 2 * (bo + ir));
+                    rr = g.rho[bo + ir];
+                }
+                rowrho[r] = rr;
+                if (SPATIAL) { rowx[r] = pr.x; rowy[r] = pr.y; }
+            }
+        }
+        // every pair of the tile has i < j < n: no masking needed
+        const bool full = (J0 >= I0 + BM) && (J0 + BN <= g.n);
+        __syncthreads();
+
+        const float w_i = roww[rl];
+        const float a_i = METRIC == 1 ? rowa[rl] : 1.f;
+        const float m2w_i = -2.f * w_i;
+        const float rho_i = rowrho[rl];
+        float x_i = 0.f, y_i = 0.f;
+        if (SPATIAL) { x_i = rowx[rl]; y_i = rowy[rl]; }
+
+        float rbest = kInf;                                // row-side minimum and its tile-local column
+        int rbest_c = -1;
+        int rthr = row_valid ? bound_of(g.best + bo + i) : (int)0x80000000;   // bits of the largest d^2 that can still serve row i
+#pragma unroll 1
+        for (int c = 0; c < kGroups; ++c) {
+            float4 nxt0 = cur0, nxt1 = cur1;
+            if (c + 1 < kGroups) {
+                nxt0 = ld_tile(src + (size_t)(2 * (c + 1)) * BM);
+                nxt1 = ld_tile(src + (size_t)(2 * (c + 1) + 1) * BM);
+            }
+            const float v[8] = {cur0.x, cur0.y, cur0.z, cur0.w, cur1.x, cur1.y, cur1.z, cur1.w};
+            const int cl0 = slice * kSliceCols + c * 8;    // tile-local first column of the group
+            // ---- every pair: d^2 and the test against the two bounds.  d^2 = a_i + a_j - 2 (g w_j) w_i, the operations
+            //      and their order as in the one-kernel sweep.  Compared as signed integers, a (rounding-level)
+            //      negative d^2, which the full treatment clamps to zero, passes every bound, as zero would.
+            float d2v[8];
+            uint32_t cand = 0;                             // bit u: column u of the group may serve this row or its column
+#pragma unroll
+            for (int q4 = 0; q4 < 2; ++q4) {
+                const float4 cw = *reinterpret_cast<const float4*>(colw + cl0 + 4 * q4);
+                const float4 cr = *reinterpret_cast<const float4*>(colrho + cl0 + 4 * q4);
+                const int4 ct = *reinterpret_cast<const int4*>(colthr + cl0 + 4 * q4);
+                float4 ca = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (METRIC == 1) ca = *reinterpret_cast<const float4*>(cola + cl0 + 4 * q4);
+                const float cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+                const float crv[4] = {cr.x, cr.y, cr.z, cr.w};
+                const float cav[4] = {ca.x, ca.y, ca.z, ca.w};
+                const int ctv[4] = {ct.x, ct.y, ct.z, ct.w};
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int u = 4 * q4 + r;
+                    const float x = v[u] * cwv[r];
+                    d2v[u] = fmaf(x, m2w_i, METRIC == 0 ? 2.f : a_i + cav[r]);
+                    // the pair can only serve the less dense of its two tokens: one bound to test, not two
+                    if (__float_as_int(d2v[u]) <= (crv[r] > rho_i ? rthr : ctv[r])) cand |= 1u << u;
+                }
+            }
+            const uint32_t live = __reduce_or_sync(0xffffffffu, cand);
+            // ---- the columns that hold a candidate: spatial radius, density order, row update, column reduction
+            if (live) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (!(live >> u & 1u)) continue;       // warp-uniform
+                    const int ce = cl0 + u;
+                    float d2 = fmaxf(d2v[u], 0.f);
+                    bool usable = true;                    // the pair may serve as (child, parent) at all
+                    if (SPATIAL) {
+                        const float dx = colx[ce] - x_i, dy = coly[ce] - y_i;
+                        usable = fmaf(dx, dx, dy * dy) <= g.tau2;
+                    }
+                    if (!full) {
+                        const int j = J0 + ce;
+                        usable = usable && j > i && j < g.n && row_valid;
+                    }
+                    if (SPATIAL || !full) d2 = usable ? d2 : kInf;
+                    // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
+                    const bool jd = colrho[ce] > rho_i;
+                    const float kr = jd ? d2 : kInf;       // j as parent candidate of i (row side)
+                    const uint32_t kc = __float_as_uint(jd ? kInf : d2);    // i as parent candidate of j (column side)
+                    if (kr < rbest) {                      // (columns come in ascending order: ties keep the lower one)
+                        rbest = kr;
+                        rbest_c = ce;
+                        rthr = min(rthr, __float_as_int(kr));
+                    }
+                    // column side: minimum over this warp's 32 rows and the lowest row that attains it; the four
+                    // warps that share the column meet in shared memory (distance first, then the lower row)
+                    const uint32_t m = __reduce_min_sync(0xffffffffu, kc);
+                    if (m < 0x7f800000u) {
+                        const uint32_t rows = __ballot_sync(0xffffffffu, kc == m);
+                        if (lane == (u & 7)) {             // (a different lane per column: the atomics of a group overlap)
+                            atomicMin(colbest + ce, ((unsigned long long)m << 32) |
+                                                        (unsigned long long)(uint32_t)(I0 + quarter * 32 + (__ffs(rows) - 1)));
+                            atomicMin(colthr + ce, (int)m);
+                        }
+                    }
+                }
+            }
+            cur0 = nxt0;
+            cur1 = nxt1;
+        }
+
+        // ---- combine the four column slices of every row and the four row quarters of every column
+        if (slice > 0) {
+            rowred[(slice - 1) * BM + rl] = rbest;
+            rowidx[(slice - 1) * BM + rl] = rbest_c;
+        }
+        __syncthreads();
+        if (slice == 0 && row_valid) {
+#pragma unroll
+            for (int q = 0; q < NS - 1; ++q) {             // ascending columns: ties keep the lower one
+                const float other = rowred[q * BM + rl];
+                if (other < rbest) { rbest = other; rbest_c = rowidx[q * BM + rl]; }
+            }
+            if (rbest_c >= 0)
+                atomicMin(g.best + bo + i, ((unsigned long long)__float_as_uint(rbest) << 32) |
+                                               (unsigned long long)(uint32_t)(J0 + rbest_c));
+        }
+        for (int ce = threadIdx.x; ce < BN; ce += kDpThreads) {
+            const unsigned long long cb = colbest[ce];
+            if (cb != ~0ull && J0 + ce < g.n) atomicMin(g.best + bo + J0 + ce, cb);
+        }
+        __syncthreads();                                   // the shared arrays are rewritten for the next tile
+    }
+}
+
+template <int BN, int METRIC, bool SPATIAL>
+int launch_dp(const GramArgs& g, const GramTiling& tl, long long total, cudaStream_t stream, bool pdl, int ctas_per_sm) {
+    cudaLaunchConfig_t cfg = {};
+    const long long ctas = (long long)ctas_per_sm * gram_num_sms();
+    cfg.gridDim = dim3((unsigned)(total < ctas ? total : ctas));
+    cfg.blockDim = dim3(kDpThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_allowed(pdl) ? 1 : 0;
+    KernelTimeScope timed("delta_pass_kernel", stream);
+    return record_cuda(cudaLaunchKernelEx(&cfg, delta_pass_kernel<BN, METRIC, SPATIAL>, g, tl, total));
+}
+
+template <int BN>
+int launch_dp_bn(const GramArgs& g, const GramTiling& tl, long long total, cudaStream_t stream, bool pdl, int cps) {
+    const bool euclid = g.metric == 1;
+    const bool spatial = g.tau2 >= 0.f && g.pos != nullptr;
+    if (spatial)
+        return euclid ? launch_dp<BN, 1, true>(g, tl, total, stream, pdl, cps)
+                      : launch_dp<BN, 0, true>(g, tl, total, stream, pdl, cps);
+    return euclid ? launch_dp<BN, 1, false>(g, tl, total, stream, pdl, cps)
+                  : launch_dp<BN, 0, false>(g, tl, total, stream, pdl, cps);
+}
+
+}  // namespace
+
+int launch_delta_pass(const GramArgs& args, const GramTiling& tiling, cudaStream_t stream, bool pdl, bool leave_room) {
+    const long long total = (long long)args.B * tiling.tiles_per_b;
+    if (total <= 0) return VITCOP_OK;
+    if (!args.gram_tiles || !args.best) return VITCOP_ERR_INVALID_ARG;
+    // four CTAs fill an SM's registers; three leave a quarter of them to a kernel that runs beside this one
+    const int cps = leave_room ? kDpCtasPerSm - 1 : kDpCtasPerSm;
+    if (tiling.BN != 256) return VITCOP_ERR_INVALID_ARG;   // (long samples always take the wide tiles)
+    return launch_dp_bn<256>(args, tiling, total, stream, pdl, cps);
+}
+
+}  // namespace vitcop

@@ -5,10 +5,12 @@
 //   1. Gram sweep, GRAM_DIAG  the diagonal tiles only: g_ii -> per-token factors (cosine: 1/sqrt(g_ii);
 //                             euclid: g_ii), from the same tensor-core arithmetic as every g_ij
 //   2. Gram sweep, GRAM_RHO   Gram tiles on the tensor cores (gram.cu); the epilogue turns each tile into
-//                             squared distances, exp(-(d/d_c)^2) and partial sums of Eq. 2 per tile
+//                             squared distances, exp(-(d/d_c)^2) and partial sums of Eq. 2 per tile, and, for
+//                             long samples, keeps the tile's Gram values in the workspace
 //   3. rho_reduce_kernel      fixed-order sum of the partials -> rho (bit-reproducible)
-//   4. Gram sweep, GRAM_DELTA the same tiles again; the epilogue keeps, per token, the nearest denser token
-//                             inside the spatial radius (Eq. 3) as a packed (d^2, j) 64-bit minimum
+//   4. delta_pass_kernel      (long samples) reads the tiles back (delta_pass.cu) and keeps, per token, the nearest
+//                             denser token inside the spatial radius (Eq. 3) as a packed (d^2, j) 64-bit minimum;
+//      Gram sweep, GRAM_DELTA (otherwise) the same tiles computed again, Eq. 3 in the epilogue
 //   5. vic_finalize_kernel    gamma = rho * delta, radix-select of the centres, pointer jumping over the
 //                             parent forest, orphan fallback, labels (Algorithm 2, steps 3-4)
 // Small problems replace 1-4 by gram_resident_kernel (gram.cu): one pass over the Gram tiles, accumulators kept in
@@ -248,10 +250,11 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
 // host side
 // ------------------------------------------------------------------------------------------------
 // Workspace of the filter: status block | row-block flags [B, ceil(n / 128)] | w | a | rho | best |
-// rho partials [B, slots, n_pad] (sized for either tile width).  The status block and the flags are zeroed at the
-// start of every call.  Words of the status block: 0 status, 2 grid barrier.
+// rho partials [B, slots, n_pad] (sized for either tile width) | Gram tiles of the density sweep (problems too large
+// for the one-kernel sweep: 4 bytes per pair of the symmetric half, tile padding included).  The status block and the
+// flags are zeroed at the start of every call.  Words of the status block: 0 status, 2 grid barrier.
 struct FilterWs {
-    size_t off_flags, off_w, off_a, off_rho, off_best, off_part, total;
+    size_t off_flags, off_w, off_a, off_rho, off_best, off_part, off_tiles, total;
     FilterWs(int B, int n) {
         size_t o = kStatusBytes;
         const size_t bn = (size_t)B * n;
@@ -262,6 +265,11 @@ struct FilterWs {
         off_best = o; o += align_up(bn * 8, 256);
         const GramTiling t = make_gram_tiling(n, 128);           // the narrow tiling has the most slots
         off_part = o; o += align_up((size_t)B * t.slots() * t.n_pad * 4, 256);
+        off_tiles = o;
+        if (gram_keeps_tiles(B, n)) {
+            const int bn = gram_pick_bn(B, n);
+            o += align_up((size_t)B * make_gram_tiling(n, bn).tiles_per_b * gram_tile_floats(bn) * 4, 256);
+        }
         total = o;
     }
 };
@@ -334,6 +342,8 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
         rc = launch_gram_resident(feat, g, make_gram_tiling(n, 128), stream);
         if (rc != VITCOP_OK) return rc;
     } else {
+        const bool keep_tiles = gram_keeps_tiles(B, n);
+        g.gram_tiles = keep_tiles ? reinterpret_cast<float*>(ws + l.off_tiles) : nullptr;
         rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
         if (rc != VITCOP_OK) return rc;
         rc = launch_gram_sweep(GRAM_RHO, feat, g, tiling, stream, true);
@@ -346,8 +356,25 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
             rc = record_cuda(cudaLaunchKernelEx(&cfg, rho_reduce_kernel, (const float*)part, n, tiling, rho, rho_user));
             if (rc != VITCOP_OK) return rc;
         }
-        rc = launch_gram_sweep(GRAM_DELTA, feat, g, tiling, stream, true);
-        if (rc != VITCOP_OK) return rc;
+        if (!keep_tiles) {
+            rc = launch_gram_sweep(GRAM_DELTA, feat, g, tiling, stream, true);
+            if (rc != VITCOP_OK) return rc;
+        }
+        // The delta pass is bound by ALU issue and by the read of the tiles, the K-norm by the read of K: given one,
+        // the pass leaves a quarter of every SM free and the K-norm, which depends on nothing in this call, runs
+        // beside it (it still waits for the pass before it ends, so the kernels behind it see both complete).
+        const bool knorm_beside = keep_tiles && knorm != nullptr;
+        if (keep_tiles) {
+            rc = launch_delta_pass(g, tiling, stream, true, knorm_beside);
+            if (rc != VITCOP_OK) return rc;
+        }
+        if (knorm_beside) {
+            rc = launch_knorm(knorm->K, knorm->B, knorm->H, knorm->d, (int64_t)knorm->H * knorm->N * knorm->d,
+                              (int64_t)knorm->N * knorm->d, knorm->d, knorm->vis_start, nullptr, knorm->Nv, knorm->score,
+                              knorm->Nv, stream, true);
+            if (rc != VITCOP_OK) return rc;
+            knorm_in_sweep = knorm->B;                     // nothing left for the launch behind vic_finalize_kernel
+        }
     }
 
     const int nc = n_centers < n ? n_centers : n;

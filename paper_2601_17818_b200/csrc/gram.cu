@@ -22,6 +22,7 @@
 
 #include <atomic>
 
+#include "async_copy.cuh"
 #include "gram.cuh"
 #include "knorm.cuh"
 
@@ -35,65 +36,10 @@ constexpr int UMMA_K = 16;
 // TMEM lane quarter).  The delta sweep's epilogue is the heavier one and gets twice the warps.
 __host__ __device__ constexpr int epi_slices(int mode) { return mode == GRAM_DELTA ? 4 : 2; }
 __host__ __device__ constexpr int gemm_threads(int mode) { return 64 + epi_slices(mode) * 128; }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded waits: after 2 s (default) give up and leave
-constexpr unsigned long long kDrainLimitNs = 20000000ull;    // bounded waits for this CTA's own copies / MMAs after giving up
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false (after raising `abort_flag`) when the time limit is hit or another role gave up.
-// limit_ns == 0 gives up at once, whatever the barrier's state (failure-handling tests use it to send one role of
-// a CTA down the give-up path while the others have work in flight).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned long long limit_ns) {
-    if (limit_ns != 0ull) {
-        if (mbar_try_wait(bar, parity)) return true;
-        const unsigned long long t0 = global_ns();
-        for (uint32_t it = 1;; ++it) {
-            if (mbar_try_wait(bar, parity)) return true;
-            if ((it & 63u) == 0u) {
-                if (*abort_flag) return false;
-                if (global_ns() - t0 > limit_ns) break;
-            }
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-// Bounded wait without side effects, used while leaving after a timeout.
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
-    const unsigned long long t0 = global_ns();
-    while (!mbar_try_wait(bar, parity))
-        if (global_ns() - t0 > kDrainLimitNs) break;
-}
-
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2) {
     asm volatile(
@@ -241,23 +187,18 @@ constexpr int kRoleLoad = 1, kRoleMma = 2, kRoleEpi = 4;
 
 template <int BN, bool SYM, bool DIAG = false>
 __device__ __forceinline__ void decode_tile(const KernelArgs& k, long long t, int& b, int& ti, int& tj) {
+    if (SYM) {
+        decode_sym_tile(k.t, t, b, ti, tj);
+        return;
+    }
     b = (int)(t / k.t.tiles_per_b);
     const int r = (int)(t - (long long)b * k.t.tiles_per_b);
     if (DIAG) {
         ti = tj = r;
         return;
     }
-    if (!SYM) {
-        ti = r / k.t.TJ;
-        tj = r - ti * k.t.TJ;
-        return;
-    }
-    constexpr int R = BN / BM;
-    int q = (int)((sqrtf(8.f * (float)r / (float)R + 1.f) - 1.f) * 0.5f);
-    while (q > 0 && R * q * (q + 1) / 2 > r) --q;
-    while (R * (q + 1) * (q + 2) / 2 <= r) ++q;
-    tj = q;
-    ti = r - R * q * (q + 1) / 2;
+    ti = r / k.t.TJ;
+    tj = r - ti * k.t.TJ;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -350,6 +291,7 @@ struct EpiCall {
     bool rho_from_part;            // GRAM_DELTA: sum rho from the density partials (and publish it from diagonal tiles)
     volatile int* abort_flag;
     unsigned long long limit_ns;   // time limit of the wait for the accumulator
+    float* store;                  // GRAM_RHO: where this tile's Gram values go (gram.cuh: layout), or null
 };
 
 // Returns true when the CTA must give up (a bounded wait expired somewhere).
@@ -507,6 +449,14 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
                     }
                 }
             } else if (MODE == GRAM_RHO) {
+                if (call.store) {
+                    // keep the Gram values for the delta pass: four columns of this thread's row per store, the
+                    // warp's 32 rows side by side
+                    float4* dst = reinterpret_cast<float4*>(call.store) + (size_t)(cl0 >> 2) * BM + rl;
+#pragma unroll
+                    for (int q4 = 0; q4 < GW / 4; ++q4)
+                        __stcs(dst + (size_t)q4 * BM, make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]));
+                }
                 // e_ij = exp(-d_ij^2 / d_c^2), Eq. 2
 #pragma unroll
                 for (int q4 = 0; q4 < GW / 4; ++q4) {
@@ -833,6 +783,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             c.rho_from_part = false;
             c.abort_flag = abort_flag;
             c.limit_ns = k.limit_of(kRoleEpi);
+            c.store = (MODE == GRAM_RHO && g.gram_tiles) ? g.gram_tiles + (size_t)t * gram_tile_floats(BN) : nullptr;
             if (epi_tile<BN, MODE, METRIC, SPATIAL, NS>(k, sm, c, ok)) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
@@ -963,11 +914,6 @@ __device__ __forceinline__ ResidentUnit decode_resident_unit(const KernelArgs& k
     return u;
 }
 
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-                 : "memory");
-}
 constexpr int kKnChunkTokens = 8;                          // tokens per chunk: 8 threads each
 constexpr int kKnBuffers = 3;
 
@@ -1190,6 +1136,7 @@ gram_resident_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             c.rho_from_part = rho_from_part;
             c.abort_flag = abort_flag;
             c.limit_ns = lim;
+            c.store = nullptr;
             return c;
         };
 
@@ -1387,9 +1334,17 @@ int launch_resident_one(const CUtensorMap& ma, const CUtensorMap& mb, const Kern
 
 }  // namespace
 
+int gram_num_sms() { return num_sms(); }
+
+unsigned long long gram_wait_limit_ns() { return g_wait_ns.load(); }
+
 void gram_set_wait_debug(unsigned long long limit_ns, int expire_roles) {
     g_wait_ns.store(limit_ns ? limit_ns : kWaitLimitNs);
     g_expire_roles.store(expire_roles & 7);
+}
+
+bool gram_keeps_tiles(int B, int n) {
+    return B > 0 && n >= kKeepTilesFromTokens && !gram_fits_resident(B, n) && gram_pick_bn(B, n) == 256;
 }
 
 int gram_pick_bn(int B, int n) {

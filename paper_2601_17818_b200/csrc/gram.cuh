@@ -35,10 +35,42 @@ inline GramTiling make_gram_tiling(int n, int BN) {
     return t;
 }
 
+// Tile t of the symmetric numbering -> (sample, row tile, column tile).
+__host__ __device__ inline void decode_sym_tile(const GramTiling& tl, long long t, int& b, int& ti, int& tj) {
+    b = (int)(t / tl.tiles_per_b);
+    const int r = (int)(t - (long long)b * tl.tiles_per_b);
+    const int R = tl.R;
+#ifdef __CUDA_ARCH__
+    int q = (int)((sqrtf(8.f * (float)r / (float)R + 1.f) - 1.f) * 0.5f);
+#else
+    int q = 0;
+#endif
+    while (q > 0 && R * q * (q + 1) / 2 > r) --q;
+    while (R * (q + 1) * (q + 2) / 2 <= r) ++q;
+    tj = q;
+    ti = r - R * q * (q + 1) / 2;
+}
+
+// The density sweep keeps the Gram values it computes: tile t (symmetric numbering, all samples) occupies
+// kGramBM * BN floats at t * kGramBM * BN, stored in groups of four columns -- element (row r, column c) at
+// ((c / 4) * kGramBM + r) * 4 + c % 4 -- so that the 32 lanes of a warp, one row each, write and read 512
+// contiguous bytes per instruction.  The delta pass (delta_pass.cu) reads them back instead of recomputing them.
+__host__ __device__ inline size_t gram_tile_floats(int BN) { return (size_t)kGramBM * BN; }
+
+// Eq. 3 needs every pair a second time, once the densities are known.  A long sample's Gram values are kept by the
+// density sweep and read back by the delta pass (4 bytes per pair against 2 D flop to recompute it); the pass is cheap
+// because most pairs fail a bound test, and the bounds only bite when every token has thousands of candidates.  For
+// shorter samples the Gram sweep is simply run again with the Eq. 3 epilogue (its loads and tensor-core work overlap
+// the density sweep's tail).  Both routes give the same bits.  Measured on one B200 (step of Stage II, microseconds):
+// 2 x 16384 tokens 1042 kept / 1135 recomputed; 8 x 2880 tokens 257 / 232; 4 x 4608 tokens 276 / 236.
+constexpr int kKeepTilesFromTokens = 8192;
+bool gram_keeps_tiles(int B, int n);
+
 // Bounded device waits of the Gram kernels: the time after which a wait gives up (0 = the default of 2 s) and, for
 // failure-handling tests, the roles whose waits give up at once (1 load warp, 2 MMA warp, 4 epilogue warps).
 // Applies to launches made after the call.
 void gram_set_wait_debug(unsigned long long limit_ns, int expire_roles);
+unsigned long long gram_wait_limit_ns();
 
 // Tile width the sweeps use for a problem: wide tiles halve the operand traffic per flop, narrow tiles fill
 // the SMs when the problem is small.
@@ -57,6 +89,7 @@ struct GramArgs {
     float* part;                // [B, slots, n_pad] rho partials  (GRAM_RHO)
     unsigned long long* best;   // [B, n] packed (d2 bits << 32 | index), ~0 = none   (GRAM_DELTA)
     float* sim_out;             // [B, row_end - row0, n]          (GRAM_SIM)
+    float* gram_tiles;          // Gram values of every visited tile, written by GRAM_RHO sweeps when not null
     float* w_out;               // [B, n] factors written by GRAM_DIAG (best, if given, is reset to ~0 as well)
     float* a_out;               // [B, n]
     float* rho_out;             // [B, n] written by the resident sweep (same memory as rho)
@@ -108,6 +141,16 @@ bool gram_resident_takes_knorm(int H, int d);
 // partials; the delta epilogue sums the partials it needs itself and re-reads the same accumulators.
 // `tiling` = make_gram_tiling(n, 128).
 int launch_gram_resident(const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream);
+
+// Eq. 3 from the Gram tiles the density sweep stored: per token the nearest denser token inside the spatial radius,
+// as a packed (d^2 bits, index) 64-bit minimum in args.best (reset to ~0 by the GRAM_DIAG sweep).  Bound by ALU issue
+// and by the read of the tiles, not by the tensor cores.  Releases its dependents at once: a kernel that does not
+// depend on it (the K-norm) can run beside it.
+// `leave_room`: occupy three quarters of every SM only.
+int launch_delta_pass(const GramArgs& args, const GramTiling& tiling, cudaStream_t stream, bool pdl, bool leave_room);
+
+// Multiprocessors of the current device.
+int gram_num_sms();
 
 // Enqueues one sweep.  `tiling` must come from make_gram_tiling(n, gram_pick_bn(B, n)) for the symmetric modes.
 int launch_gram_sweep(int mode, const void* feat, const GramArgs& args, const GramTiling& tiling, cudaStream_t stream,

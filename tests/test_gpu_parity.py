@@ -434,6 +434,23 @@ def test_filter_resident_shapes(B, n, metric, check):
         check_vic_sample(f[b], p[b], metric, d_c, w.tau, nc, g.rho[b], g.delta2[b], g.parent[b], g.label[b])
 
 
+# Long samples (8192 tokens and more) keep the Gram tiles of the density sweep and run Eq. 3 as a separate pass over
+# them: a ragged length (tiles that straddle the diagonal and the end of the sample), both metrics, with and
+# without the spatial test.  Small feature width: the oracle's pairwise work stays cheap.
+@pytest.mark.parametrize("n,metric,tau", [(8200, 0, 0.6), (8321, 1, 0.6), (8200, 0, -1.0), (8192, 0, 0.25)])
+def test_filter_long_sample_delta_pass(n, metric, tau):
+    w = dataclasses.replace(W.workload("c4"), B=1, D=64, dup_rate=0.3)
+    f = W.make_features(w, n=n, B=1)
+    p = W.make_positions(w, n)[:1]
+    d_c = w.d_c if metric == 0 else 40.0                 # (euclid: 1 % of the tokens have ten times the norm)
+    nc = n // 20
+    g = gpu_filter(f, p, metric, d_c, tau, nc)
+    assert g.status == vb.OK and np.all(g.n_clusters == nc)
+    rep = []
+    check_vic_sample(f[0], p[0], metric, d_c, tau, nc, g.rho[0], g.delta2[0], g.parent[0], g.label[0], rep)
+    print("filter long sample", n, metric, tau, rep)
+
+
 def test_filter_edge_cases():
     w = W.workload("tiny")
     # identical tokens: one cluster led by token 0
