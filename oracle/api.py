@@ -256,6 +256,25 @@ def cls_saliency(q_bits: np.ndarray, K_bits: np.ndarray, scale: float):
     return S, float(c.value)
 
 
+def kproj_knorm(hidden_bits: np.ndarray, W_bits: np.ndarray, H: int, d: int, cos: Optional[np.ndarray] = None,
+                sin: Optional[np.ndarray] = None, position: Optional[np.ndarray] = None):
+    """K = W_k t per head (+ rotary embedding), rounded to bf16, and its Eq. 4 norm, for one sample.
+
+    hidden bf16 bits [N, Dh], W bf16 bits [H*d, Dh], cos / sin float64 [n_pos, d/2] or None, position int32 [N] or None.
+    Returns (K float64 [H, N, d] before rounding, K bf16 bits [H, N, d], score float64 [N])."""
+    h, W = _u16(hidden_bits), _u16(W_bits)
+    N, Dh = h.shape
+    assert W.shape == (H * d, Dh)
+    c = None if cos is None else np.ascontiguousarray(cos, dtype=np.float64)
+    s = None if sin is None else np.ascontiguousarray(sin, dtype=np.float64)
+    pos = None if position is None else np.ascontiguousarray(position, dtype=np.int32)
+    K64 = np.empty((H, N, d), dtype=np.float64)
+    Kb = np.empty((H, N, d), dtype=np.uint16)
+    score = np.empty(N, dtype=np.float64)
+    lib().oracle_kproj_knorm(_p(h), _p(W), N, Dh, H, d, _p(c), _p(s), _p(pos), _p(K64), _p(Kb), _p(score))
+    return K64, Kb, score
+
+
 def flops_layer(N: float, d: float) -> float:
     return float(lib().oracle_flops_layer(C.c_double(N), C.c_double(d)))
 

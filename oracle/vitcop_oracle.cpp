@@ -428,6 +428,62 @@ void oracle_cls_saliency(const uint16_t* q, const uint16_t* K, int H, int M, int
     if (cls_out) *cls_out = total[0];
 }
 
+// ---------------------------------------------------------------------------------------------
+// O9. The K vectors of Eq. 4 at their source: K^(h)_i = W_k^(h) t_i for every head (one row of W per output
+//   feature, as a linear layer stores it), optionally rotated by rotary position embedding (pairs (e, e + d/2) of a
+//   head turned by the angle whose cosine / sine the tables give at the token's position), and the K-norm of Eq. 4
+//   taken on the bf16 values a K cache would hold.  One sample.
+//   hidden [N, Dh] and W [H * d, Dh] are bf16 bit patterns; cos_tab / sin_tab [n_pos, d / 2] doubles or NULL (no
+//   rotation); position [N] (NULL: token index).  Outputs: K64 [H, N, d] doubles (before rounding), K_bf16 [H, N, d]
+//   bit patterns (round to nearest even), score [N] = sqrt(sum over heads and elements of the rounded values squared).
+// ---------------------------------------------------------------------------------------------
+static uint16_t double_to_bf16_rne(double v) {
+    float f = static_cast<float>(v);                        // fp64 -> fp32 -> bf16: the double rounding can differ from a
+    uint32_t u;                                             // direct one only on exact ties of the second step, which the
+    std::memcpy(&u, &f, sizeof u);                          // first step's 29 discarded bits make vanishingly rare
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x40);   // NaN stays NaN
+    const uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return static_cast<uint16_t>(u >> 16);
+}
+
+void oracle_kproj_knorm(const uint16_t* hidden, const uint16_t* W, int N, int Dh, int H, int d, const double* cos_tab,
+                        const double* sin_tab, const int32_t* position, double* K64, uint16_t* K_bf16, double* score) {
+    const int half = d / 2;
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < N; ++t) {
+        std::vector<double> row(static_cast<size_t>(H) * d);
+        for (int c = 0; c < H * d; ++c) {
+            double acc = 0.0;
+            for (int k = 0; k < Dh; ++k)
+                acc += bf16_to_double(hidden[static_cast<size_t>(t) * Dh + k]) * bf16_to_double(W[static_cast<size_t>(c) * Dh + k]);
+            row[c] = acc;
+        }
+        if (cos_tab && sin_tab) {
+            const int p = position ? position[t] : t;
+            for (int h = 0; h < H; ++h)
+                for (int e = 0; e < half; ++e) {
+                    const double a = row[h * d + e], b = row[h * d + e + half];
+                    const double c = cos_tab[static_cast<size_t>(p) * half + e], s = sin_tab[static_cast<size_t>(p) * half + e];
+                    row[h * d + e] = a * c - b * s;
+                    row[h * d + e + half] = b * c + a * s;
+                }
+        }
+        double acc = 0.0;
+        for (int h = 0; h < H; ++h)
+            for (int e = 0; e < d; ++e) {
+                const double v = row[h * d + e];
+                const size_t o = (static_cast<size_t>(h) * N + t) * d + e;
+                const uint16_t r = double_to_bf16_rne(v);
+                if (K64) K64[o] = v;
+                if (K_bf16) K_bf16[o] = r;
+                const double q = bf16_to_double(r);
+                acc += q * q;
+            }
+        score[t] = std::sqrt(acc);
+    }
+}
+
 // Cost model of Appendix E.  Eq. 7: FLOPs of one transformer layer on a sequence of N tokens, hidden size d.
 double oracle_flops_layer(double N, double d) { return 4.0 * N * N * d + 16.0 * N * d * d; }
 

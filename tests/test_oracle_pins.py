@@ -694,3 +694,62 @@ def test_cost_model_closed_forms():
     # Eq. 10 equals one minus the layer average of Eq. 8 over m
     avg = sum(oracle.visual_tokens_at_layer(l, m, *p) for l in range(1, 33)) / (32 * m)
     assert abs(oracle.cr_int(*p) - (1 - avg)) < 1e-15
+
+
+# =============================================================================== O9: K projection + K-norm
+def test_kproj_identity_weights_reduce_to_knorm():
+    # W = I (H * d == Dh): K is the hidden row cut into heads, so the score is Eq. 4 of that tensor
+    rng = np.random.default_rng(7)
+    N, H, d = 9, 4, 8
+    hid = bf16(rng.standard_normal((N, H * d)))
+    W_id = bf16(np.eye(H * d))
+    K64, Kb, score = oracle.kproj_knorm(hid, W_id, H, d)
+    as_K = np.ascontiguousarray(hid.reshape(N, H, d).transpose(1, 0, 2))          # [H, N, d]
+    assert np.array_equal(Kb, as_K)
+    assert np.array_equal(K64, W.bf16_bits_to_f32(as_K).astype(np.float64))
+    assert np.array_equal(score, oracle.knorm(as_K[None], 0, N)[0])
+
+
+def test_kproj_one_hot_weights_pick_hidden_elements():
+    rng = np.random.default_rng(8)
+    N, Dh, H, d = 5, 24, 2, 4
+    hid = bf16(rng.standard_normal((N, Dh)))
+    pick = rng.permutation(Dh)[: H * d]
+    Wm = np.zeros((H * d, Dh), dtype=np.float32)
+    Wm[np.arange(H * d), pick] = -2.0                       # scaling by a power of two is exact
+    K64, Kb, score = oracle.kproj_knorm(hid, bf16(Wm), H, d)
+    want = -2.0 * W.bf16_bits_to_f32(hid).astype(np.float64)[:, pick].reshape(N, H, d).transpose(1, 0, 2)
+    assert np.array_equal(K64, want)
+    np.testing.assert_allclose(score, np.sqrt((want ** 2).sum((0, 2))), rtol=1e-14)
+
+
+def test_kproj_matches_a_matmul_and_rounds_to_nearest_even():
+    rng = np.random.default_rng(9)
+    N, Dh, H, d = 7, 40, 3, 8
+    hid, Wk = bf16(rng.standard_normal((N, Dh))), bf16(rng.standard_normal((H * d, Dh)) * 0.2)
+    K64, Kb, score = oracle.kproj_knorm(hid, Wk, H, d)
+    ref = W.bf16_bits_to_f32(hid).astype(np.float64) @ W.bf16_bits_to_f32(Wk).astype(np.float64).T      # [N, H*d]
+    np.testing.assert_allclose(K64, ref.reshape(N, H, d).transpose(1, 0, 2), rtol=1e-13, atol=1e-13)
+    assert np.array_equal(Kb, W.f32_to_bf16_bits(K64.astype(np.float32)))                               # the repo's own rounding
+    Kr = W.bf16_bits_to_f32(Kb).astype(np.float64)
+    np.testing.assert_allclose(score, np.sqrt((Kr ** 2).sum((0, 2))), rtol=1e-14)
+    assert np.array_equal(score, oracle.knorm(Kb[None], 0, N)[0])                                       # Eq. 4 of the rounded K
+
+
+def test_kproj_rotary_embedding_quarter_turn_and_norm_invariance():
+    rng = np.random.default_rng(10)
+    N, Dh, H, d = 6, 16, 2, 8
+    hid, Wk = bf16(rng.standard_normal((N, Dh))), bf16(rng.standard_normal((H * d, Dh)))
+    plain, _, _ = oracle.kproj_knorm(hid, Wk, H, d)
+    # a quarter turn at every position: (a, b) -> (-b, a) for the pairs (e, e + d/2)
+    cos, sin = np.zeros((N, d // 2)), np.ones((N, d // 2))
+    rot, _, _ = oracle.kproj_knorm(hid, Wk, H, d, cos, sin)
+    assert np.array_equal(rot[..., : d // 2], -plain[..., d // 2:]) and np.array_equal(rot[..., d // 2:], plain[..., : d // 2])
+    # any angles: the norm before rounding is unchanged; positions select the table row
+    ang = rng.random((50, d // 2)) * 6.0
+    position = rng.integers(0, 50, size=N).astype(np.int32)
+    rot, _, _ = oracle.kproj_knorm(hid, Wk, H, d, np.cos(ang), np.sin(ang), position)
+    np.testing.assert_allclose((rot ** 2).sum((0, 2)), (plain ** 2).sum((0, 2)), rtol=1e-12)
+    a, b = plain[1, 3, 2], plain[1, 3, 2 + d // 2]
+    c, s_ = np.cos(ang[position[3], 2]), np.sin(ang[position[3], 2])
+    assert abs(rot[1, 3, 2] - (a * c - b * s_)) < 1e-12 and abs(rot[1, 3, 2 + d // 2] - (b * c + a * s_)) < 1e-12
