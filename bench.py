@@ -490,6 +490,9 @@ class Bench:
                                                          for v in kernels.values()),
                            "event_bracket_overhead_us": bracket_us}
 
+        # K-norm at the source of K: the key projection with the norm in its epilogue (no separate read of K) -------
+        res["kproj_knorm"] = self.kproj(res["isolated"]["knorm_kernel"]["us_per_launch"])
+
         # end to end through the public API with host buffers --------------------------------------------------
         res["e2e"] = self.e2e(e2e_steps, pruned_per_step)
 
@@ -556,6 +559,34 @@ class Bench:
         units = algorithmic_units(w, 0, B * n, int(nk[0].sum()))["compact_kernel"][1]
         out["compact_kernel"] = {"us_per_launch": us, "copies": R, **self.roofline_entry("hbm", units, us)}
         del ins, outs
+        torch.cuda.empty_cache()
+        return out
+
+    def kproj(self, knorm_us):
+        """vitcop_kproj_knorm at the workload's shapes (layer input -> K of all heads with rotary embedding + Eq. 4 of
+        the visual span), against the tensor-core peak; beside it what the stand-alone K-norm of that K costs."""
+        w, sc, torch, vb, dev = self.w, self.sc, self.torch, self.vb, self.dev
+        g = torch.Generator(device=dev).manual_seed(0)
+        Wk = (torch.randn((w.H * w.d, w.Dh), device=dev, generator=g) / w.Dh ** 0.5).to(torch.bfloat16)
+        inv = 1.0 / (10000.0 ** (torch.arange(w.d // 2, device=dev) / (w.d // 2)))
+        ang = torch.arange(w.N, device=dev)[:, None] * inv[None, :]
+        cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+        K_out = torch.empty((w.B, w.H, w.N, w.d), dtype=torch.bfloat16, device=dev)
+        score = torch.empty((w.B, w.Nv), dtype=torch.float32, device=dev)
+        ws = vb.alloc_workspace(vb.OP_KPROJ, device=dev, B=w.B, H=w.H, N=w.N, d=w.d)
+        fn = lambda: vb.vitcop_kproj_knorm(sc.hidden, Wk, w.H, w.d, K_out, ws, vis_start=w.vis_start, score=score,
+                                           rope_cos=cos, rope_sin=sin)
+        t = self.timed(fn, 10, 3)
+        us = float(np.median(t) * 1e3)
+        flop = 2.0 * w.B * w.N * w.Dh * w.H * w.d
+        tf = flop / (us * 1e-6) / 1e12
+        out = {"us_median": us, "flop": flop, "achieved": tf, "unit": "TFLOP/s", "peak": self.peaks["bf16_tflops"],
+               "frac": tf / self.peaks["bf16_tflops"], "peak_source": self.peaks["source"] + " burst",
+               "knorm_standalone_us": knorm_us,
+               "note": "GEMM [B*N, Dh] x [Dh, H*d] + rotary embedding + bf16 K + Eq. 4 in the epilogue; the stand-alone "
+                       "K-norm (knorm_standalone_us, the separate read of K) is what a pruning step saves when K comes "
+                       "from this call"}
+        del Wk, K_out
         torch.cuda.empty_cache()
         return out
 
@@ -667,7 +698,8 @@ def run_ours(args):
                                 l2="flushed (512 MiB memset) before every timed step", sharding="replicas only"),
             "clocks": head["clocks"], "e2e": head["e2e"], "gpu_launches": head["gpu_launches_per_step"] * args.steps,
             "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"], "kernels": head["kernels"],
-            "isolated": head["isolated"], "schedule": head["schedule"], "plain_step0": head["plain_step0"],
+            "isolated": head["isolated"], "kproj_knorm": head["kproj_knorm"], "schedule": head["schedule"],
+            "plain_step0": head["plain_step0"],
             "stage2_as_two_calls_us": head["stage2_as_two_calls_us"],
             "us_per_step_median": head["us_per_step_median"], "other_workloads": others,
         }

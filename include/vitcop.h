@@ -53,6 +53,7 @@ extern "C" {
 #define VITCOP_OP_SALIENCY    6   /* vitcop_cls_saliency: B = images, H = heads, N = keys per head (M) */
 #define VITCOP_OP_MERGE       7   /* vitcop_merge_clusters: Nv = Nv_cap, N = Mcap */
 #define VITCOP_OP_COLLAB_STEP 8   /* vitcop_collaborative_step */
+#define VITCOP_OP_KPROJ       9   /* vitcop_kproj_knorm: B, H, N, d */
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* vitcop_status_string(int status);
@@ -290,6 +291,27 @@ int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh,
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
 int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, int d, float scale,
                         float* saliency, float* cls_self, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- K-norm at the source of K
+ * Eq. 4 needs the K vectors "from the LLM's attention module".  This call produces them: K^(h)_t = W_k^(h) x_t for
+ * every head as one bf16 GEMM on the tensor cores, optional rotary position embedding, K written in bf16 in the cache
+ * layout the other calls read, and the K-norm of the visual span from the same pass, so that the pruning step needs
+ * no second read of K (its largest byte term).  The norm is taken on the bf16 values that are stored (what
+ * vitcop_knorm_score would compute from K_out), squares and sums in fp32; a rotation does not change it beyond
+ * rounding (Eq. 4 is rotation invariant).
+ *   hidden        bf16 [B, N, Dh]     layer input (Dh multiple of 64)
+ *   W_k           bf16 [H * d, Dh]    key projection, one row per output feature (d multiple of 32)
+ *   rope_cos/sin  fp32 [n_pos, d / 2] or both NULL: pairs (e, e + d / 2) of a head are turned by the angle of the
+ *                 token's position, (a, b) -> (a cos - b sin, b cos + a sin); needs d in {64, 128, 256}
+ *   position_ids  int32 [B, N] or NULL (position = token index); clamped to [0, n_pos)
+ *   K_out         bf16 [B, H, N, d] out
+ *   score         fp32 [B, Nv] out, optional: Eq. 4 of tokens vis_start .. vis_start + Nv - 1
+ *   workspace     vitcop_workspace_bytes(VITCOP_OP_KPROJ, B, H, N, d, ..) bytes
+ * Errors: INVALID_ARG, UNSUPPORTED (divisibility, alignment), WORKSPACE, CUDA. */
+int vitcop_kproj_knorm(const void* hidden, const void* W_k, int B, int N, int Dh, int H, int d,
+                       const float* rope_cos, const float* rope_sin, const int32_t* position_ids, int n_pos,
+                       void* K_out, int vis_start, int Nv, float* score,
+                       void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------- schedule and cost model (host arithmetic)
  * Algorithm 1 prunes to floor(m * pi) tokens per stage (pi relative to the ORIGINAL m visual tokens); Appendix E

@@ -18,7 +18,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvitcop.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA, ERR_TIMEOUT = range(7)
-OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY, OP_MERGE, OP_COLLAB_STEP = range(9)
+(OP_FILTER, OP_KNORM, OP_SELECT, OP_COMPACT, OP_PRUNE_STEP, OP_SIMILARITY, OP_SALIENCY, OP_MERGE, OP_COLLAB_STEP,
+ OP_KPROJ) = range(10)
 MAX_VISUAL_TOKENS = 16384
 
 EXPORTS = [
@@ -27,7 +28,7 @@ EXPORTS = [
     "vitcop_compact_kv", "vitcop_prune_step", "vitcop_kernel_timing_begin", "vitcop_kernel_timing_end",
     "vitcop_prune_step_static", "vitcop_merge_clusters", "vitcop_cls_saliency", "vitcop_stage_count",
     "vitcop_flops_layer", "vitcop_visual_tokens_at_layer", "vitcop_flops_total", "vitcop_cr_int",
-    "vitcop_collaborative_step", "vitcop_set_wait_limit",
+    "vitcop_collaborative_step", "vitcop_set_wait_limit", "vitcop_kproj_knorm",
 ]
 
 
@@ -97,6 +98,7 @@ def lib() -> C.CDLL:
                                                 i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                                 vp, vp, sz, vp]
         L.vitcop_set_wait_limit.argtypes = [C.c_ulonglong, i32]
+        L.vitcop_kproj_knorm.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp, sz, vp]
         L.vitcop_kernel_timing_begin.argtypes = []
         L.vitcop_kernel_timing_end.argtypes = [C.POINTER(KernelTime), i32, C.POINTER(C.c_int)]
         for name in EXPORTS:
@@ -270,6 +272,20 @@ def vitcop_cls_saliency(q_cls, K, scale: float, saliency, workspace, cls_self=No
                                    _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "vitcop_cls_saliency")
     return saliency
+
+
+def vitcop_kproj_knorm(hidden, W_k, H: int, d: int, K_out, workspace, vis_start: int = 0, score=None, rope_cos=None,
+                       rope_sin=None, position_ids=None):
+    """K = W_k x per head (+ rotary embedding) in bf16 [B,H,N,d] and Eq. 4 of the visual span from the same pass."""
+    B, N, Dh = hidden.shape
+    assert W_k.shape == (H * d, Dh) and K_out.shape == (B, H, N, d)
+    Nv = 0 if score is None else score.shape[1]
+    n_pos = 0 if rope_cos is None else rope_cos.shape[0]
+    rc = lib().vitcop_kproj_knorm(_ptr(hidden), _ptr(W_k), B, N, Dh, H, d, _ptr(rope_cos), _ptr(rope_sin),
+                                  _ptr(position_ids), n_pos, _ptr(K_out), int(vis_start), Nv, _ptr(score),
+                                  _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "vitcop_kproj_knorm")
+    return K_out
 
 
 def vitcop_stage_count(m: int, pi: float) -> int:

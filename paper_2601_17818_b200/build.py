@@ -13,7 +13,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 BUILD_DIR = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libvitcop.so")
-SOURCES = ["api.cu", "knorm.cu", "select.cu", "compact.cu", "filter.cu", "gram.cu", "delta_pass.cu", "merge.cu", "saliency.cu",
+SOURCES = ["api.cu", "knorm.cu", "select.cu", "compact.cu", "filter.cu", "gram.cu", "delta_pass.cu", "kproj.cu", "merge.cu", "saliency.cu",
            "schedule.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]

@@ -187,7 +187,7 @@ int vitcop_kernel_timing_end(vitcop_kernel_time* out, int capacity, int* count) 
 }
 
 int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, int Dh, size_t* bytes) {
-    (void)d; (void)Dh;
+    (void)Dh;
     if (!bytes || B < 0 || Nv < 0 || D < 0) return VITCOP_ERR_INVALID_ARG;
     switch (op) {
         case VITCOP_OP_FILTER: *bytes = filter_workspace_bytes(B, Nv, D); return VITCOP_OK;
@@ -202,6 +202,10 @@ int vitcop_workspace_bytes(int op, int B, int H, int N, int d, int Nv, int D, in
         case VITCOP_OP_MERGE:
             if (N < 0) return VITCOP_ERR_INVALID_ARG;
             *bytes = merge_workspace_bytes(B, Nv, N);
+            return VITCOP_OK;
+        case VITCOP_OP_KPROJ:
+            if (H < 0 || N < 0 || d < 0) return VITCOP_ERR_INVALID_ARG;
+            *bytes = kproj_workspace_bytes(B, N, H, d);
             return VITCOP_OK;
         case VITCOP_OP_SALIENCY:
             if (H < 0 || N < 0) return VITCOP_ERR_INVALID_ARG;
@@ -409,6 +413,28 @@ int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, i
     int rc = reset_status(workspace, s);
     if (rc != VITCOP_OK) return rc;
     return launch_cls_saliency(q_cls, K, B, H, M, d, scale, saliency, cls_self, workspace, s);
+}
+
+int vitcop_kproj_knorm(const void* hidden, const void* W_k, int B, int N, int Dh, int H, int d, const float* rope_cos,
+                       const float* rope_sin, const int32_t* position_ids, int n_pos, void* K_out, int vis_start, int Nv,
+                       float* score, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hidden || !W_k || !K_out || B < 0 || N < 0 || Dh < 0 || H < 0 || d < 0 || Nv < 0 || vis_start < 0)
+        return VITCOP_ERR_INVALID_ARG;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr)) return VITCOP_ERR_INVALID_ARG;
+    if (rope_cos && n_pos <= 0) return VITCOP_ERR_INVALID_ARG;
+    if (score && vis_start + (int64_t)Nv > N) return VITCOP_ERR_INVALID_ARG;
+    if (Dh % 64 || d % 32 || !aligned16(hidden) || !aligned16(W_k) || !aligned16(K_out)) return VITCOP_ERR_UNSUPPORTED;
+    if (rope_cos && ((d != 64 && d != 128 && d != 256) || !aligned16(rope_cos) || !aligned16(rope_sin)))
+        return VITCOP_ERR_UNSUPPORTED;
+    if ((int64_t)B * N > 0x7fffffff || (int64_t)H * d > 0x7fffffff || B > 65535) return VITCOP_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < kproj_workspace_bytes(B, N, H, d) || !aligned256(workspace))
+        return VITCOP_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = reset_status(workspace, s);
+    if (rc != VITCOP_OK) return rc;
+    if (B == 0 || N == 0 || H == 0 || d == 0 || Dh == 0) return VITCOP_OK;
+    return launch_kproj_knorm(hidden, W_k, B, N, Dh, H, d, rope_cos, rope_sin, position_ids, n_pos, K_out, vis_start,
+                              score ? Nv : 0, score, workspace, s);
 }
 
 int vitcop_prune_step_static(const void* hidden, const void* K, const void* V, int B, int H, int N, int d, int Dh,

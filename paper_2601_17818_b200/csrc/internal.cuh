@@ -70,6 +70,11 @@ int launch_merge(const void* hidden, int B, int N, int Dh, int vis_start, const 
                  cudaStream_t stream);
 size_t merge_workspace_bytes(int B, int Nv_cap, int Mcap);
 
+size_t kproj_workspace_bytes(int B, int N, int H, int d);
+int launch_kproj_knorm(const void* hidden, const void* W, int B, int N, int Dh, int H, int d, const float* cos_tab,
+                       const float* sin_tab, const int32_t* position, int n_pos, void* K_out, int vis_start, int Nv,
+                       float* score, void* workspace, cudaStream_t stream);
+
 size_t saliency_workspace_bytes(int B, int H, int M);
 int launch_cls_saliency(const void* q, const void* K, int B, int H, int M, int d, float scale, float* saliency,
                         float* cls_self, void* workspace, cudaStream_t stream);

@@ -121,6 +121,14 @@ def test_argument_validation_of_the_wider_entry_points(L):
     assert L.vitcop_collaborative_step(*args(D=72)) == vb.ERR_UNSUPPORTED
     assert L.vitcop_collaborative_step(*args(wsb=64)) == vb.ERR_WORKSPACE
     assert L.vitcop_collaborative_step(*args(B=65536, wsb=1 << 40)) == vb.ERR_UNSUPPORTED      # as its sibling calls
+    # K projection: weights required, cos and sin together, rotation only for head sizes whose halves are chunk-aligned
+    kp = lambda hid=fake, W=fake, Dh=64, d=64, cos=null, sin=null, npos=0, wsb=1 << 24: (hid, W, 1, 8, Dh, 2, d, cos, sin, null, npos, b, 0, 4, fake, ws, wsb, null)
+    assert L.vitcop_kproj_knorm(*kp(W=null)) == vb.ERR_INVALID_ARG
+    assert L.vitcop_kproj_knorm(*kp(cos=fake)) == vb.ERR_INVALID_ARG
+    assert L.vitcop_kproj_knorm(*kp(Dh=72)) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_kproj_knorm(*kp(d=32, cos=fake, sin=fake, npos=8)) == vb.ERR_UNSUPPORTED
+    assert L.vitcop_kproj_knorm(*kp(wsb=64)) == vb.ERR_WORKSPACE
+    assert vb.vitcop_workspace_bytes(vb.OP_KPROJ, B=2, H=4, N=100, d=128) >= 2 * 2 * 100 * 4
     assert vb.vitcop_workspace_bytes(vb.OP_COLLAB_STEP, B=2, Nv=100, D=64) > vb.vitcop_workspace_bytes(vb.OP_FILTER, B=2, Nv=100, D=64)
     assert vb.vitcop_workspace_bytes(vb.OP_MERGE, B=2, Nv=100, N=10) >= 256 + 2 * 100 * 2
     assert vb.vitcop_workspace_bytes(vb.OP_SALIENCY, B=2, H=4, N=33) >= 2 * 4 * 33 * 4

@@ -135,3 +135,90 @@ def test_stage_one_chain():
         oracle_band_check(want_S, keeps[b], k1, SAL_RTOL, largest=True)
         assert np.array_equal(keeps[b], oracle.select_plain(g_S[b].astype(np.float64), k1, True))
         assert np.array_equal(got[b], feat[b][keeps[b]]) and int(olen[b]) == k1
+
+
+# ======================================================================================= K projection + K-norm
+# The call writes K in bf16 and reports Eq. 4 of exactly those values.  What is checked:
+#   K:      |gpu - oracle fp64| <= one bf16 spacing of the value (2^-8 relative: the rounding step, taken on an fp32
+#           accumulator here and on the fp64 value in the oracle, may fall either way near a tie) + the fp32
+#           accumulation error, bounded by 2e-6 |x_t| |w_c|; and nearly all elements round to the oracle's bits;
+#   score:  relative 1e-5 against Eq. 4 of the K the call wrote (the definition of what it reports), and relative
+#           1e-4 against the oracle's own rounded K (a few roundings that fell the other way move it by ~1e-5).
+KPROJ_ULP = 2.0 ** -8
+
+
+def _kproj_case(B, N, Dh, H, d, rope, vis_start, Nv, rows=None, seed=0):
+    rng = np.random.default_rng(seed)
+    hid = W.f32_to_bf16_bits(rng.standard_normal((B, N, Dh)).astype(np.float32))
+    Wk = W.f32_to_bf16_bits((rng.standard_normal((H * d, Dh)) / np.sqrt(Dh)).astype(np.float32))
+    n_pos = N + 5
+    cos = sin = pos = None
+    if rope:
+        inv = 1.0 / (10000.0 ** (np.arange(d // 2) / (d // 2)))
+        ang = np.arange(n_pos)[:, None] * inv[None, :]
+        cos, sin = np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+        pos = rng.integers(0, n_pos, size=(B, N)).astype(np.int32)
+    K_out = torch.zeros((B, H, N, d), dtype=torch.bfloat16, device=DEV)
+    score = torch.full((B, Nv), -7.0, dtype=torch.float32, device=DEV)
+    ws = vb.alloc_workspace(vb.OP_KPROJ, B=B, H=H, N=N, d=d)
+    t = lambda a: None if a is None else torch.from_numpy(a).to(DEV)
+    vb.vitcop_kproj_knorm(vb.bf16_tensor(hid), vb.bf16_tensor(Wk), H, d, K_out, ws, vis_start=vis_start, score=score,
+                          rope_cos=t(cos), rope_sin=t(sin), position_ids=t(pos))
+    assert vb.vitcop_poll_status(ws) == vb.OK
+    g_K, g_score = vb.bf16_bits(K_out), score.cpu().numpy()
+    # Eq. 4 of the K that was written, every token of the span
+    own = oracle.knorm(g_K, vis_start, Nv)
+    assert np.all(rel_err(g_score, own) <= KNORM_RTOL), rel_err(g_score, own).max()
+    # against the oracle's projection: all rows of small cases, a seeded sample of rows otherwise
+    xf, wf = W.bf16_bits_to_f32(hid).astype(np.float64), W.bf16_bits_to_f32(Wk).astype(np.float64)
+    wn = np.sqrt((wf * wf).sum(1)).reshape(H, 1, d)
+    same = total = 0
+    for b in range(B):
+        sel = np.arange(N) if rows is None else np.sort(rng.permutation(N)[:rows])
+        K64, Kb, o_score = oracle.kproj_knorm(np.ascontiguousarray(hid[b, sel]), Wk, H, d,
+                                              None if cos is None else cos.astype(np.float64),
+                                              None if sin is None else sin.astype(np.float64),
+                                              None if pos is None else np.ascontiguousarray(pos[b, sel]))
+        if pos is None and rope:
+            raise AssertionError
+        got = W.bf16_bits_to_f32(g_K[b][:, sel]).astype(np.float64)
+        xn = np.sqrt((xf[b, sel] ** 2).sum(1)).reshape(1, -1, 1)
+        assert np.all(np.abs(got - K64) <= KPROJ_ULP * np.abs(K64) + 2e-6 * xn * wn)
+        same += int((g_K[b][:, sel] == Kb).sum())
+        total += Kb.size
+        in_span = (sel >= vis_start) & (sel < vis_start + Nv)
+        if in_span.any():
+            assert np.all(rel_err(g_score[b, sel[in_span] - vis_start], o_score[in_span]) <= 1e-4)
+    assert same >= 0.97 * total, (same, total)
+
+
+@pytest.mark.parametrize("B,N,Dh,H,d,rope", [(2, 77, 128, 3, 64, False), (1, 300, 256, 4, 128, True),
+                                              (3, 130, 192, 2, 256, True), (2, 64, 64, 5, 32, False),
+                                              (2, 200, 320, 6, 64, True), (1, 129, 64, 1, 128, False)])
+def test_kproj_knorm_small(B, N, Dh, H, d, rope):
+    _kproj_case(B, N, Dh, H, d, rope, vis_start=min(5, N - 1), Nv=max(1, N - 9), seed=N)
+
+
+def test_kproj_knorm_identity_weights_and_text_only_span():
+    # W = I: K is the hidden row cut into heads, bit for bit, and the score is Eq. 4 of the input
+    rng = np.random.default_rng(3)
+    B, N, H, d = 2, 70, 2, 64
+    hid = W.f32_to_bf16_bits(rng.standard_normal((B, N, H * d)).astype(np.float32))
+    K_out = torch.zeros((B, H, N, d), dtype=torch.bfloat16, device=DEV)
+    score = torch.zeros((B, N), dtype=torch.float32, device=DEV)
+    ws = vb.alloc_workspace(vb.OP_KPROJ, B=B, H=H, N=N, d=d)
+    eye = W.f32_to_bf16_bits(np.eye(H * d, dtype=np.float32))
+    vb.vitcop_kproj_knorm(vb.bf16_tensor(hid), vb.bf16_tensor(eye), H, d, K_out, ws, score=score)
+    want = np.ascontiguousarray(hid.reshape(B, N, H, d).transpose(0, 2, 1, 3))
+    assert np.array_equal(vb.bf16_bits(K_out), want)
+    assert np.all(rel_err(score.cpu().numpy(), oracle.knorm(want, 0, N)) <= KNORM_RTOL)
+    vb.vitcop_kproj_knorm(vb.bf16_tensor(hid), vb.bf16_tensor(eye), H, d, K_out, ws)          # no span: K only
+    assert vb.vitcop_poll_status(ws) == vb.OK and np.array_equal(vb.bf16_bits(K_out), want)
+
+
+@pytest.mark.parametrize("name", ["c1", "c4"])
+def test_kproj_knorm_workload_shapes(name):
+    """The projection at the shapes of a benchmark workload (c1: 10240 tokens x 4096 -> 32 heads of 128); the oracle
+    checks a seeded sample of token rows, Eq. 4 of the written K is checked on every token."""
+    w = W.workload(name)
+    _kproj_case(w.B, w.N, w.Dh, w.H, w.d, True, w.vis_start, w.Nv, rows=6, seed=1)
