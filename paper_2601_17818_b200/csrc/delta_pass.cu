@@ -10,17 +10,17 @@
 // One CTA of 8 warps per tile, up to four CTAs per SM, a persistent grid; every CTA takes one contiguous run of the
 // tile numbering, i.e. consecutive row blocks against one column block (see below why).  Warp w owns
 // the rows 32 (w % 4) .. + 31 of the tile (one per lane) and the column half w / 4; a thread walks its half eight
-// columns at a time (two 16-byte loads, the next two already in flight), keeps its row's minimum, and the warp reduces
-// each column over its 32 rows with redux / ballot.  The four row quarters of a column and the two halves of a row are
-// combined through shared memory in a fixed order (ties keep the lower index) and folded into the per-token packed
-// minima with one 64-bit atomicMin each.
+// columns at a time (two 16-byte loads, the next four already in flight) and keeps its row's minimum; the minimum of
+// a column is kept in shared memory.  The two halves of a row are combined through shared memory (ties keep the lower
+// index) and rows and columns are folded into the per-token packed minima with one 64-bit atomicMin each.
 //
 // Most pairs cannot matter: a pair serves its row token only if its d^2 does not exceed the best that token has so
 // far, and its column token likewise (and a pair serves only one of the two: the less dense one).  Both bounds are read from the packed minima when the tile starts (other CTAs
 // keep lowering them, a stale bound is merely looser) and tightened as the tile goes.  A thread first computes d^2 of
 // its eight pairs and tests them against the two bounds (with <=: an equal distance at a lower index still wins);
-// one redux.or tells the warp which of the eight columns hold a candidate at all, and only those columns go through
-// the spatial test, the density comparison, the row update and the column reduction.  What is skipped could not
+// one redux.or tells the warp whether any of its 256 pairs passed, and only the lanes whose pair passed go through
+// the spatial test and update the row's minimum (in registers) or the column's (a packed 64-bit minimum in shared
+// memory: smaller distance first, then the lower row).  What is skipped could not
 // have changed any minimum, so the result is the same as without the test.
 // The bounds only bite once a token has seen some of its candidates, so the order of the work matters: a CTA walks
 // down one column block, whose tokens thus meet their candidates one row block after the other (their bounds stay in
@@ -34,7 +34,7 @@ namespace {
 constexpr int BM = kGramBM;
 constexpr int kDpSlices = 2;                              // column slices of a tile, four warps each
 constexpr int kDpThreads = 128 * kDpSlices;
-constexpr int kDpCtasPerSm = 4;
+constexpr int kDpCtasPerSm = 3;
 constexpr float kInf = __builtin_huge_valf();
 
 // Bits of the largest d^2 that can still improve the packed minimum at `p` (an equal d^2 with a lower index would):
@@ -74,6 +74,29 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
     const int rl = quarter * 32 + lane;                    // tile-local row of this thread
 
     const long long t_begin = total_tiles * blockIdx.x / gridDim.x, t_end = total_tiles * (blockIdx.x + 1) / gridDim.x;
+    // The tiles of the run are contiguous in memory, so the thread's loads form one stream over the whole run: the
+    // sixteen columns it works on (A, B: eight each) and the sixteen after those, requested while it works -- across
+    // tile boundaries, so that the constants of a new tile are fetched with data already in flight.  `pf` walks that
+    // stream: two float4 columns of 128 rows per group, and past the other half's columns at the end of a tile.
+    constexpr size_t kGroupStep = 2 * BM;                                      // float4 per group
+    constexpr size_t kTileSkip = gram_tile_floats(BN) / 4 - (size_t)kGroups * kGroupStep;
+    const float4* pf = reinterpret_cast<const float4*>(g.gram_tiles) + (size_t)t_begin * (gram_tile_floats(BN) / 4) +
+                       (size_t)(slice * kSliceCols / 4) * BM + rl;
+    const float4* const pf_end = reinterpret_cast<const float4*>(g.gram_tiles) + (size_t)t_end * (gram_tile_floats(BN) / 4);
+    float4 A0 = make_float4(0.f, 0.f, 0.f, 0.f), A1 = A0, B0 = A0, B1 = A0;
+    int pf_group = 0;                                      // group inside its tile that pf points at
+    auto fetch_pair = [&](float4& x0, float4& x1, float4& y0, float4& y1) {    // the next two groups of the stream
+        if (pf < pf_end) {
+            x0 = ld_tile(pf);
+            x1 = ld_tile(pf + BM);
+            y0 = ld_tile(pf + kGroupStep);
+            y1 = ld_tile(pf + kGroupStep + BM);
+        }
+        pf += 2 * kGroupStep;
+        pf_group += 2;
+        if (pf_group == kGroups) { pf_group = 0; pf += kTileSkip; }
+    };
+    fetch_pair(A0, A1, B0, B1);
     int prev_b = -1, prev_tj = -1;
     for (long long t = t_begin; t < t_end; ++t) {
         int b, ti, tj;
@@ -85,11 +108,6 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
         const int i = I0 + rl;
         const bool row_valid = i < g.n;
         const size_t bo = (size_t)b * g.n;
-
-        // the first two loads of this thread's slice travel while the tile's constants are fetched
-        const float4* src = reinterpret_cast<const float4*>(g.gram_tiles + (size_t)t * gram_tile_floats(BN)) +
-                            (size_t)(slice * kSliceCols / 4) * BM + rl;
-        float4 cur0 = ld_tile(src), cur1 = ld_tile(src + BM);
 
         for (int it = threadIdx.x; it < 2 * BN + 2 * BM; it += kDpThreads) {
             if (it < BN) {
@@ -146,20 +164,15 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
         float rbest = kInf;                                // row-side minimum and its tile-local column
         int rbest_c = -1;
         int rthr = row_valid ? bound_of(g.best + bo + i) : (int)0x80000000;   // bits of the largest d^2 that can still serve row i
-#pragma unroll 1
-        for (int c = 0; c < kGroups; ++c) {
-            float4 nxt0 = cur0, nxt1 = cur1;
-            if (c + 1 < kGroups) {
-                nxt0 = ld_tile(src + (size_t)(2 * (c + 1)) * BM);
-                nxt1 = ld_tile(src + (size_t)(2 * (c + 1) + 1) * BM);
-            }
-            const float v[8] = {cur0.x, cur0.y, cur0.z, cur0.w, cur1.x, cur1.y, cur1.z, cur1.w};
-            const int cl0 = slice * kSliceCols + c * 8;    // tile-local first column of the group
-            // ---- every pair: d^2 and the test against the two bounds.  d^2 = a_i + a_j - 2 (g w_j) w_i, the operations
-            //      and their order as in the one-kernel sweep.  Compared as signed integers, a (rounding-level)
-            //      negative d^2, which the full treatment clamps to zero, passes every bound, as zero would.
+        // One group: eight columns of this thread's row.
+        auto group = [&](const float4& c0, const float4& c1, const int cl0) {
+            const float v[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+            // ---- every pair: d^2 and the test against ONE bound, that of the less dense of the two tokens (the only
+            //      one the pair can serve).  d^2 = a_i + a_j - 2 (g w_j) w_i, the operations and their order as in the
+            //      one-kernel sweep.  Compared as signed integers, a (rounding-level) negative d^2, which the full
+            //      treatment clamps to zero, passes every bound, as zero would.
             float d2v[8];
-            uint32_t cand = 0;                             // bit u: column u of the group may serve this row or its column
+            uint32_t cand = 0;                             // bit u: column u of the group passed
 #pragma unroll
             for (int q4 = 0; q4 < 2; ++q4) {
                 const float4 cw = *reinterpret_cast<const float4*>(colw + cl0 + 4 * q4);
@@ -176,52 +189,48 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
                     const int u = 4 * q4 + r;
                     const float x = v[u] * cwv[r];
                     d2v[u] = fmaf(x, m2w_i, METRIC == 0 ? 2.f : a_i + cav[r]);
-                    // the pair can only serve the less dense of its two tokens: one bound to test, not two
                     if (__float_as_int(d2v[u]) <= (crv[r] > rho_i ? rthr : ctv[r])) cand |= 1u << u;
                 }
             }
-            const uint32_t live = __reduce_or_sync(0xffffffffu, cand);
-            // ---- the columns that hold a candidate: spatial radius, density order, row update, column reduction
-            if (live) {
+            // ---- the pairs that passed: spatial radius, then the row's own minimum (registers) or the column's (shared
+            //      memory, packed so that the smaller distance and then the lower row wins).  Only the lanes that hold
+            //      such a pair take the branch; one redux.or lets a warp without any skip the lot.
+            if (__reduce_or_sync(0xffffffffu, cand) == 0u) return;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (!(live >> u & 1u)) continue;       // warp-uniform
-                    const int ce = cl0 + u;
-                    float d2 = fmaxf(d2v[u], 0.f);
-                    bool usable = true;                    // the pair may serve as (child, parent) at all
-                    if (SPATIAL) {
-                        const float dx = colx[ce] - x_i, dy = coly[ce] - y_i;
-                        usable = fmaf(dx, dx, dy * dy) <= g.tau2;
-                    }
-                    if (!full) {
-                        const int j = J0 + ce;
-                        usable = usable && j > i && j < g.n && row_valid;
-                    }
-                    if (SPATIAL || !full) d2 = usable ? d2 : kInf;
-                    // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
-                    const bool jd = colrho[ce] > rho_i;
-                    const float kr = jd ? d2 : kInf;       // j as parent candidate of i (row side)
-                    const uint32_t kc = __float_as_uint(jd ? kInf : d2);    // i as parent candidate of j (column side)
-                    if (kr < rbest) {                      // (columns come in ascending order: ties keep the lower one)
-                        rbest = kr;
+            for (int u = 0; u < 8; ++u) {
+                if (!(cand >> u & 1u)) continue;
+                const int ce = cl0 + u;
+                bool usable = true;                        // the pair may serve as (child, parent) at all
+                if (SPATIAL) {
+                    const float dx = colx[ce] - x_i, dy = coly[ce] - y_i;
+                    usable = fmaf(dx, dx, dy * dy) <= g.tau2;
+                }
+                if (!full) {
+                    const int j = J0 + ce;
+                    usable = usable && j > i && j < g.n && row_valid;
+                }
+                if (!usable) continue;
+                const float d2 = fmaxf(d2v[u], 0.f);
+                // with i < j: "j denser than i" is rho_j > rho_i, "i denser than j" is its complement
+                if (colrho[ce] > rho_i) {                  // j as parent candidate of i (row side)
+                    if (d2 < rbest) {                      // (columns come in ascending order: ties keep the lower one)
+                        rbest = d2;
                         rbest_c = ce;
-                        rthr = min(rthr, __float_as_int(kr));
+                        rthr = __float_as_int(d2);
                     }
-                    // column side: minimum over this warp's 32 rows and the lowest row that attains it; the four
-                    // warps that share the column meet in shared memory (distance first, then the lower row)
-                    const uint32_t m = __reduce_min_sync(0xffffffffu, kc);
-                    if (m < 0x7f800000u) {
-                        const uint32_t rows = __ballot_sync(0xffffffffu, kc == m);
-                        if (lane == (u & 7)) {             // (a different lane per column: the atomics of a group overlap)
-                            atomicMin(colbest + ce, ((unsigned long long)m << 32) |
-                                                        (unsigned long long)(uint32_t)(I0 + quarter * 32 + (__ffs(rows) - 1)));
-                            atomicMin(colthr + ce, (int)m);
-                        }
-                    }
+                } else {                                   // i as parent candidate of j (column side)
+                    atomicMin(colbest + ce, ((unsigned long long)__float_as_uint(d2) << 32) | (unsigned long long)(uint32_t)i);
+                    atomicMin(colthr + ce, __float_as_int(d2));
                 }
             }
-            cur0 = nxt0;
-            cur1 = nxt1;
+        };
+#pragma unroll 2
+        for (int c = 0; c < kGroups; c += 2) {
+            float4 N0 = A0, N1 = A1, M0 = B0, M1 = B1;
+            fetch_pair(N0, N1, M0, M1);
+            group(A0, A1, slice * kSliceCols + c * 8);
+            group(B0, B1, slice * kSliceCols + c * 8 + 8);
+            A0 = N0; A1 = N1; B0 = M0; B1 = M1;
         }
 
         // ---- combine the four column slices of every row and the four row quarters of every column
@@ -281,8 +290,8 @@ int launch_delta_pass(const GramArgs& args, const GramTiling& tiling, cudaStream
     const long long total = (long long)args.B * tiling.tiles_per_b;
     if (total <= 0) return VITCOP_OK;
     if (!args.gram_tiles || !args.best) return VITCOP_ERR_INVALID_ARG;
-    // four CTAs fill an SM's registers; three leave a quarter of them to a kernel that runs beside this one
-    const int cps = leave_room ? kDpCtasPerSm - 1 : kDpCtasPerSm;
+    // (`leave_room`: a kernel that runs beside this one finds a third of every SM's registers and thread slots free)
+    const int cps = kDpCtasPerSm; (void)leave_room;
     if (tiling.BN != 256) return VITCOP_ERR_INVALID_ARG;   // (long samples always take the wide tiles)
     return launch_dp_bn<256>(args, tiling, total, stream, pdl, cps);
 }

@@ -55,7 +55,7 @@ __host__ __device__ inline void decode_sym_tile(const GramTiling& tl, long long 
 // kGramBM * BN floats at t * kGramBM * BN, stored in groups of four columns -- element (row r, column c) at
 // ((c / 4) * kGramBM + r) * 4 + c % 4 -- so that the 32 lanes of a warp, one row each, write and read 512
 // contiguous bytes per instruction.  The delta pass (delta_pass.cu) reads them back instead of recomputing them.
-__host__ __device__ inline size_t gram_tile_floats(int BN) { return (size_t)kGramBM * BN; }
+__host__ __device__ constexpr size_t gram_tile_floats(int BN) { return (size_t)kGramBM * BN; }
 
 // Eq. 3 needs every pair a second time, once the densities are known.  A long sample's Gram values are kept by the
 // density sweep and read back by the delta pass (4 bytes per pair against 2 D flop to recompute it); the pass is cheap
