@@ -39,7 +39,7 @@ HEADLINE = "c4"
 ALL_WORKLOADS = ("c0", "c1", "c2", "c3", "c4")
 L2_BYTES = 126 << 20
 KERNEL_SOURCE = {"knorm_kernel": "knorm.cu", "compact_kernel": "compact.cu", "gram_tc_kernel<rho>": "gram.cu",
-                 "gram_tc_kernel<delta>": "gram.cu", "gram_resident_kernel": "gram.cu"}
+                 "gram_tc_kernel<delta>": "gram.cu", "gram_resident_kernel": "gram.cu", "delta_pass_kernel": "delta_pass.cu"}
 
 
 def measured_peaks():
@@ -337,7 +337,9 @@ def algorithmic_units(w, s, vis_in, kept):
     if s == 0:
         sweep = w.B * w.Nv * (w.Nv + 1) * w.D
         u.update({"gram_resident_kernel": ("tensor", sweep), "gram_tc_kernel<rho>": ("tensor", sweep),
-                  "gram_tc_kernel<delta>": ("tensor", sweep)})
+                  "gram_tc_kernel<delta>": ("tensor", sweep),
+                  # reads the stored Gram value of every pair of the symmetric half (diagonal included) once: 4 bytes
+                  "delta_pass_kernel": ("hbm", w.B * w.Nv * (w.Nv + 1) // 2 * 4)})
     return u
 
 
@@ -562,7 +564,7 @@ class Bench:
         torch.cuda.empty_cache()
         return out
 
-    def kproj(self, knorm_us):
+    def kproj(self, knorm_us, reps=10, warm=3):
         """vitcop_kproj_knorm at the workload's shapes (layer input -> K of all heads with rotary embedding + Eq. 4 of
         the visual span), against the tensor-core peak; beside it what the stand-alone K-norm of that K costs."""
         w, sc, torch, vb, dev = self.w, self.sc, self.torch, self.vb, self.dev
@@ -576,7 +578,7 @@ class Bench:
         ws = vb.alloc_workspace(vb.OP_KPROJ, device=dev, B=w.B, H=w.H, N=w.N, d=w.d)
         fn = lambda: vb.vitcop_kproj_knorm(sc.hidden, Wk, w.H, w.d, K_out, ws, vis_start=w.vis_start, score=score,
                                            rope_cos=cos, rope_sin=sin)
-        t = self.timed(fn, 10, 3)
+        t = self.timed(fn, reps, warm)
         us = float(np.median(t) * 1e3)
         flop = 2.0 * w.B * w.N * w.Dh * w.H * w.d
         tf = flop / (us * 1e-6) / 1e12
@@ -668,6 +670,8 @@ def run_ours(args):
         for _ in range(args.warmup + args.steps):
             flush.zero_()
             b.sc.run()
+        flush.zero_()
+        b.kproj(0.0, reps=1, warm=0)                       # the key projection with the K-norm in its epilogue, once
         torch.cuda.synchronize()
         print(json.dumps({"profile_run": w.name, "steps": args.steps, "warmup": args.warmup}))
         return
