@@ -124,10 +124,10 @@ def oracle_sample(w, per_step_seconds):
     """A bounded sample of the workload for the CPU oracle: (workload to run, number of sequences, description).
 
     Sequences are independent, so the sample is the first few of them; a sequence of the long-video workload
-    alone costs about half a minute of pairwise fp64 work, so where even one sequence exceeds the bound it is cut to
+    alone costs about a quarter of a minute of pairwise fp64 work, so where even one sequence exceeds the bound it is cut to
     its first 4096 visual tokens (budgets and centre count scaled alike) -- the pairwise work per token then is a
     quarter of the full length's, which the description says."""
-    cost = {"c0": 0.05, "c1": 0.05, "c2": 1.5, "c3": 4.0, "c4": 50.0}.get(w.name, 0.05)   # seconds per sequence, roughly
+    cost = {"c0": 0.02, "c1": 0.02, "c2": 0.6, "c3": 1.0, "c4": 16.0}.get(w.name, 0.05)   # seconds per sequence on 16 cores, roughly
     if cost <= per_step_seconds:
         nseq = int(max(1, min(w.B, per_step_seconds // cost, 4)))
         return w, nseq, f"the first {nseq} of {w.B} sequences of workload {w.name}, whole schedule"
