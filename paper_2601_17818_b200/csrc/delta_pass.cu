@@ -195,9 +195,11 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
             // ---- the pairs that passed: spatial radius, then the row's own minimum (registers) or the column's (shared
             //      memory, packed so that the smaller distance and then the lower row wins).  Only the lanes that hold
             //      such a pair take the branch; one redux.or lets a warp without any skip the lot.
-            if (__reduce_or_sync(0xffffffffu, cand) == 0u) return;
+            const uint32_t live = __reduce_or_sync(0xffffffffu, cand);     // columns in which some lane's pair passed
+            if (live == 0u) return;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
+                if (!(live >> u & 1u)) continue;           // warp-uniform: a column nobody needs costs one branch
                 if (!(cand >> u & 1u)) continue;
                 const int ce = cl0 + u;
                 bool usable = true;                        // the pair may serve as (child, parent) at all
