@@ -501,7 +501,7 @@ class Bench:
         # CPU oracle beside it -----------------------------------------------------------------------------------
         res["cpu_baseline"] = None
         if cpu_seconds > 0:
-            ob = OracleBench(w, per_step_seconds=max(cpu_seconds, 60.0 if w.name == "c4" else cpu_seconds))
+            ob = OracleBench(w, per_step_seconds=max(cpu_seconds, 20.0 if w.name == "c4" else cpu_seconds))
             v, secs, passes = ob.run_for(cpu_seconds)
             res["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ob.cores, "kind": "oracle",
                                    "sample": f"{ob.sample}, {passes} pass(es) in {secs:.1f} s"}
