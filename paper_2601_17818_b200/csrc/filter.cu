@@ -42,6 +42,7 @@ __global__ void rho_reduce_kernel(const float* __restrict__ part, int n, GramTil
 // Centres, forest roots and labels: one CTA per sample.
 // ------------------------------------------------------------------------------------------------
 constexpr int kFinThreads = 1024;
+constexpr int kFinIters = VITCOP_MAX_VISUAL_TOKENS / kFinThreads;      // tokens per thread at the largest sample
 
 // Shared memory: keys[n] (uint64; later reused as next[n] int32), isc[n] (uint8), centres[nc] (int32).
 __global__ void __launch_bounds__(kFinThreads)
@@ -56,6 +57,7 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
     int32_t* centres = reinterpret_cast<int32_t*>(fin_smem + (size_t)n * 8 + (((size_t)n + 15) & ~(size_t)15));
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_sums[32];
+    __shared__ uint32_t cnt[kFinIters * 32];               // one count per (iteration, warp)
     __shared__ uint32_t s_digit, s_krem, s_whole;
     __shared__ unsigned long long orph_best[kFinThreads];
     __shared__ int orph_list[kFinThreads];
@@ -144,27 +146,57 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
         }
         T = prefix;
     }
-    // ---- centre flags + ascending centre list
+    // ---- centre flags + ascending centre list.  Token i = it * 1024 + tid; ranks in index order come from one count
+    //      per (iteration, warp), scanned once for the whole sample, plus the lane's position in its warp's ballot:
+    //      first among the keys equal to the cut (ties -> lower index), then among the centres.
     {
-        uint32_t eq_running = 0, c_running = 0;
-        for (int base = 0; base < n; base += kFinThreads) {
-            const int i = base + tid;
-            const unsigned long long key = i < n ? keys[i] : ~0ull;
+        uint32_t eq_mask = 0, f_mask = 0;                  // bit it: this thread's token of iteration it is ... / is a centre
+        const int iters = (n + kFinThreads - 1) / kFinThreads;          // <= kFinIters
+        const uint32_t lane_below = (1u << lane) - 1u;
+        const bool cut = nc > 0 && nc < n;
+        if (cut) {
+            for (int it = 0; it < iters; ++it) {
+                const int i = it * kFinThreads + tid;
+                const bool eq = i < n && keys[i] == T;
+                const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+                if (eq) eq_mask |= 1u << it;
+                if (lane == 0) cnt[it * 32 + warp] = __popc(bal);
+            }
+            __syncthreads();
+            uint32_t total;
+            const uint32_t excl = block_exclusive_sum(tid < iters * 32 ? cnt[tid] : 0u, warp_sums, total);
+            if (tid < iters * 32) cnt[tid] = excl;
+            __syncthreads();
+        }
+        for (int it = 0; it < iters; ++it) {
+            const int i = it * kFinThreads + tid;
             bool f;
             if (nc <= 0) f = false;
             else if (nc >= n) f = i < n;
             else {
-                const bool eq = i < n && key == T;
-                uint32_t eq_total;
-                const uint32_t eq_rank = eq_running + block_prefix_count(eq, warp_sums, eq_total);
-                eq_running += eq_total;
-                f = i < n && (key < T || (eq && eq_rank < krem));
+                const bool eq = (eq_mask >> it & 1u) != 0;
+                const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+                const uint32_t eq_rank = cnt[it * 32 + warp] + __popc(bal & lane_below);
+                f = i < n && (keys[i] < T || (eq && eq_rank < krem));
             }
-            uint32_t c_total;
-            const uint32_t r = c_running + block_prefix_count(f, warp_sums, c_total);
-            c_running += c_total;
+            if (f) f_mask |= 1u << it;
             if (i < n) isc[i] = f ? 1 : 0;
-            if (f && r < (uint32_t)nc) centres[r] = i;
+        }
+        __syncthreads();                                   // cnt is reused
+        for (int it = 0; it < iters; ++it) {
+            const uint32_t bal = __ballot_sync(0xffffffffu, (f_mask >> it & 1u) != 0);
+            if (lane == 0) cnt[it * 32 + warp] = __popc(bal);
+        }
+        __syncthreads();
+        uint32_t total;
+        const uint32_t excl = block_exclusive_sum(tid < iters * 32 ? cnt[tid] : 0u, warp_sums, total);
+        if (tid < iters * 32) cnt[tid] = excl;
+        __syncthreads();
+        for (int it = 0; it < iters; ++it) {
+            const bool f = (f_mask >> it & 1u) != 0;
+            const uint32_t bal = __ballot_sync(0xffffffffu, f);
+            const uint32_t r = cnt[it * 32 + warp] + __popc(bal & lane_below);
+            if (f && r < (uint32_t)nc) centres[r] = it * kFinThreads + tid;
         }
     }
     __syncthreads();   // keys are dead from here on; nxt aliases them
@@ -195,7 +227,10 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
         label[i] = isc[root] ? root : -1 - root;
     }
     __syncthreads();
-    if (nc > 0) {
+    int any_surplus = 0;                                   // a root that is neither a centre nor below one
+    for (int i = tid; i < n; i += kFinThreads) any_surplus |= (!isc[i] && nxt[i] == i) ? 1 : 0;
+    any_surplus = __syncthreads_or(any_surplus);
+    if (nc > 0 && any_surplus) {
         // Surplus orphans (roots that are not centres) are rare but each needs its distance to every centre: they
         // are listed, kFinThreads tokens at a time, and the (orphan, centre) pairs are spread over all warps; the
         // nearest centre wins through a packed minimum (distance bits, then the lower centre rank).

@@ -110,6 +110,30 @@ __device__ __forceinline__ uint32_t block_prefix_count(bool flag, uint32_t* warp
     __syncthreads();
     return (warp == 0 ? 0u : base) + before;
 }
+
+// Exclusive prefix sum of one value per thread over a CTA of 1024 threads, in thread order; `total` receives the CTA-wide sum.
+__device__ __forceinline__ uint32_t block_exclusive_sum(uint32_t v, uint32_t* warp_sums, uint32_t& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    uint32_t w = warp_sums[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, w, off);
+        if (lane >= off) w += t;
+    }
+    total = __shfl_sync(0xffffffffu, w, 31);
+    const uint32_t base = warp == 0 ? 0u : __shfl_sync(0xffffffffu, w, warp - 1);
+    __syncthreads();
+    return base + incl - v;
+}
+
 #endif
 
 }  // namespace vitcop

@@ -74,31 +74,10 @@ constexpr int kMaxSeg = 1024;
 constexpr int kSegTok = 16;                               // tokens per thread: VITCOP_MAX_VISUAL_TOKENS / kSelThreads
 constexpr uint32_t kSegDone = 0xFFFFFFFFu;
 constexpr int kRankWork = 64;                             // rank search when sum |C_c|^2 <= kRankWork * n ...
+constexpr int kRankWorkLong = 16;                         // ... (long samples: a CTA's 1024 threads share all of it) ...
+constexpr int kRankLongTokens = 8192;
 constexpr int kRankMaxSize = 2048;                        // ... and no searched cluster is larger than this
 constexpr int kRadixMinTokens = 4096;                     // below this a sort beats the radix passes (fewer barriers)
-
-// Exclusive prefix sum of one value per thread over the CTA, in thread order; `total` receives the CTA-wide sum.
-__device__ __forceinline__ uint32_t block_exclusive_sum(uint32_t v, uint32_t* warp_sums, uint32_t& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t incl = v;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += t;
-    }
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    uint32_t w = warp_sums[lane];
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, w, off);
-        if (lane >= off) w += t;
-    }
-    total = __shfl_sync(0xffffffffu, w, 31);
-    const uint32_t base = warp == 0 ? 0u : __shfl_sync(0xffffffffu, w, warp - 1);
-    __syncthreads();
-    return base + incl - v;
-}
 
 // Writes the tokens whose flag is set in keepf[0..n) to keep_idx in ascending order (every thread scans a run of
 // consecutive tokens, one block-wide scan places the runs); returns their number.
@@ -250,7 +229,8 @@ __device__ __forceinline__ bool select_quota_by_cluster(const float* score, cons
         const uint32_t o = block_exclusive_sum(size, warp_sums, total);   // its barriers publish misc as well
         if (tid < (int)n_seg) offs[tid] = o;
     }
-    const bool by_rank = misc[3] == 0 && (unsigned long long)misc[2] <= (unsigned long long)kRankWork * (unsigned)n;
+    const bool by_rank = misc[3] == 0 && (unsigned long long)misc[2] <=
+                                             (unsigned long long)(n > kRankLongTokens ? kRankWorkLong : kRankWork) * (unsigned)n;
     const uint32_t range_lo = misc[0], range_hi = misc[1];
     if (!by_rank && n <= kRadixMinTokens) return false;    // uniform; nothing has been written yet
     __syncthreads();
