@@ -478,10 +478,6 @@ class Bench:
 
         # single-kernel calls without brackets (what matters for kernels of a few tens of microseconds) ---------
         res["isolated"] = self.isolated(vis_in, kept)
-        for name, iso in res["isolated"].items():
-            k0 = f"{name}@0"
-            if k0 in kernels and "bound" in kernels[k0] and "us_per_launch" in iso and name != "knorm_kernel":
-                pass
         # the roofline of the kernel with the largest share of the step
         d = kernels[dom[0]]
         res["roofline"] = {"kernel": dom[0].split("@")[0], "stage": int(dom[0].split("@")[1]),
@@ -494,6 +490,9 @@ class Bench:
 
         # K-norm at the source of K: the key projection with the norm in its epilogue (no separate read of K) -------
         res["kproj_knorm"] = self.kproj(res["isolated"]["knorm_kernel"]["us_per_launch"])
+
+        # the operators beside the pruning step: cluster merge (Eq. 6), [CLS] saliency (Eq. 1) ---------------------
+        res["beside_the_step"] = self.beside_the_step()
 
         # end to end through the public API with host buffers --------------------------------------------------
         res["e2e"] = self.e2e(e2e_steps, pruned_per_step)
@@ -561,6 +560,54 @@ class Bench:
         units = algorithmic_units(w, 0, B * n, int(nk[0].sum()))["compact_kernel"][1]
         out["compact_kernel"] = {"us_per_launch": us, "copies": R, **self.roofline_entry("hbm", units, us)}
         del ins, outs
+        torch.cuda.empty_cache()
+        return out
+
+    def beside_the_step(self):
+        """Cluster merge (Eq. 6) on Stage II's own labels and keep mask, and [CLS] saliency (Eq. 1) over the workload's
+        heads with n + 1 keys, as stand-alone calls by the back-to-back protocol, against the copy bandwidth."""
+        w, sc, torch, vb, dev = self.w, self.sc, self.torch, self.vb, self.dev
+        B, n = w.B, w.Nv
+        out = {}
+        # ---- merge: reads the hidden row of every visual token that was not kept, writes one row per cluster
+        score = torch.empty((B, n), dtype=torch.float32, device=dev)
+        vb.vitcop_knorm_score(sc.K[0], w.vis_start, n, score)
+        kidx = torch.empty((B, n), dtype=torch.int32, device=dev)
+        nk = torch.empty((B,), dtype=torch.int32, device=dev)
+        km = torch.empty((B, n), dtype=torch.uint8, device=dev)
+        vb.vitcop_select(score, n, w.budgets[0], kidx, nk, vb.alloc_workspace(vb.OP_SELECT, device=dev, B=B, Nv=n),
+                         label=sc.label, keep_mask=km)
+        M = w.n_centers
+        hbytes = B * w.N * w.Dh * 2
+        R = int(min(16, max(2, -(-3 * L2_BYTES // hbytes))))
+        hids = [sc.hidden] + [sc.hidden.clone() for _ in range(R - 1)]
+        ml = [torch.empty((B, M), dtype=torch.int32, device=dev) for _ in range(R)]
+        mc = [torch.empty((B, M), dtype=torch.int32, device=dev) for _ in range(R)]
+        nm = [torch.empty((B,), dtype=torch.int32, device=dev) for _ in range(R)]
+        mr = [torch.empty((B, M, w.Dh), dtype=torch.bfloat16, device=dev) for _ in range(R)]
+        ws = [vb.alloc_workspace(vb.OP_MERGE, device=dev, B=B, Nv=n, N=M) for _ in range(R)]
+        us, copies = self.back_to_back(lambda i: (lambda: vb.vitcop_merge_clusters(
+            hids[i % R], w.vis_start, n, sc.label, km, ml[i % R], mc[i % R], nm[i % R], ws[i % R], merged=mr[i % R])),
+            hbytes)
+        merged_rows, dropped = int(nm[0].sum()), B * n - int(nk.sum())
+        units = dropped * w.Dh * 2 + merged_rows * (w.Dh * 2 + 8) + B * n * 5
+        out["merge_clusters"] = {"us_per_call": us, "copies": copies, "rows_read": dropped, "rows_written": merged_rows,
+                                 **self.roofline_entry("hbm", units, us)}
+        del hids, mr
+        # ---- saliency: reads every key of every head once
+        g = torch.Generator(device=dev).manual_seed(1)
+        kbytes = B * w.H * (n + 1) * w.d * 2
+        R = int(min(48, max(2, -(-3 * L2_BYTES // kbytes))))
+        Kc = (torch.randn((B, w.H, n + 1, w.d), device=dev, generator=g)).to(torch.bfloat16)
+        Ks = [Kc] + [Kc.clone() for _ in range(R - 1)]
+        q = torch.randn((B, w.H, w.d), device=dev, generator=g).to(torch.bfloat16)
+        sal = [torch.empty((B, n), dtype=torch.float32, device=dev) for _ in range(R)]
+        wss = [vb.alloc_workspace(vb.OP_SALIENCY, device=dev, B=B, H=w.H, N=n + 1) for _ in range(R)]
+        us, copies = self.back_to_back(lambda i: (lambda: vb.vitcop_cls_saliency(q, Ks[i % R], w.d ** -0.5, sal[i % R],
+                                                                                wss[i % R])), kbytes)
+        out["cls_saliency"] = {"us_per_call": us, "copies": copies, "heads": w.H, "keys": n + 1,
+                               **self.roofline_entry("hbm", kbytes + B * n * 4, us)}
+        del Ks
         torch.cuda.empty_cache()
         return out
 
@@ -702,7 +749,8 @@ def run_ours(args):
                                 l2="flushed (512 MiB memset) before every timed step", sharding="replicas only"),
             "clocks": head["clocks"], "e2e": head["e2e"], "gpu_launches": head["gpu_launches_per_step"] * args.steps,
             "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"], "kernels": head["kernels"],
-            "isolated": head["isolated"], "kproj_knorm": head["kproj_knorm"], "schedule": head["schedule"],
+            "isolated": head["isolated"], "kproj_knorm": head["kproj_knorm"],
+            "beside_the_step": head["beside_the_step"], "schedule": head["schedule"],
             "plain_step0": head["plain_step0"],
             "stage2_as_two_calls_us": head["stage2_as_two_calls_us"],
             "us_per_step_median": head["us_per_step_median"], "other_workloads": others,

@@ -2,43 +2,117 @@
 // averaged into one representative row.
 //
 // Two kernels on one stream:
-//   merge_plan_kernel   one CTA per sample: sorts the (label, token index) pairs of the non-elite tokens in shared
-//                       memory, which lays every cluster's members out contiguously in ascending token order; the
-//                       clusters that have members are numbered in ascending label order (ordered ballot/popc
-//                       compaction of the run heads) and the member list goes to the workspace
-//   merge_rows_kernel   one CTA per (merged row, sample, 512-byte slice of the hidden row): its eight warps stream
-//                       the members' row slices with 128-bit loads (member r goes to warp r mod 8) and the eight
+//   merge_plan_kernel   one CTA per sample: gathers the non-elite tokens in token order and sorts them by label with
+//                       a stable radix sort in shared memory, which lays every cluster's members out contiguously
+//                       in ascending token order; the clusters that have members are numbered in ascending label
+//                       order (ordered ballot/popc compaction of the run heads) and the member list goes to the
+//                       workspace
+//   merge_rows_kernel   one CTA per (merged row, sample, 512-byte slice of the hidden row): its four warps stream
+//                       the members' row slices with 128-bit loads (member r goes to warp r mod 4) and the four
 //                       fp32 partial sums are added in warp order, a fixed order (bit-reproducible).  Only rows
 //                       that are averaged are read.
 #include <cuda_bf16.h>
 
-#include "block_sort.cuh"
 #include "internal.cuh"
 
 namespace vitcop {
 namespace {
 
 constexpr int kPlanThreads = 1024;
-constexpr int kRowsThreads = 256;
+constexpr int kPlanWarps = kPlanThreads / 32;
+constexpr int kRowsThreads = 128;
+constexpr int kPlanItems = VITCOP_MAX_VISUAL_TOKENS / kPlanThreads;   // rows of 32 entries a warp walks at most
+constexpr int kDigitBits = 7, kDigits = 1 << kDigitBits;
+static_assert(kDigits * kPlanWarps == 4 * kPlanThreads, "four counters per thread in the scan");
+// The counter of (digit d, warp w) sits at w * kCntStride + d: the leaders of a row (one warp, distinct digits) and
+// the four counters a thread scans (one digit, consecutive warps) both spread over the banks.
+constexpr int kCntStride = kDigits + 2;
+constexpr int kCntEntries = kPlanWarps * kCntStride;
 
-// Loads the keys (label << 32 | index) of the non-elite tokens, ~0 for everything else, and sorts them.
-template <int E>
-__device__ void sort_members(const int32_t* __restrict__ label, const uint8_t* __restrict__ keep_mask, int n, int T,
-                             unsigned long long* comp) {
-    unsigned long long r[E];
-    const int t = threadIdx.x;
+// Every array of the planner is walked the same way: warp w owns the entries [w * 32 E, (w + 1) * 32 E), E =
+// ceil(count / 1024), and takes them 32 at a time, lane by lane (coalesced, no bank conflicts, and entry order is
+// (warp, row, lane) order, so that ballots and one scan over the 32 warp totals give stable positions).  The walks are
+// rolled loops on purpose: the kernel runs once per call on a handful of SMs, so every instruction it executes is
+// fetched cold, and a loop body fetched once beats sixteen unrolled copies.
+
+// Exclusive prefix of one value per warp (uniform inside the warp) over the CTA's 32 warps; `total` = the sum.
+__device__ __forceinline__ uint32_t warp_totals_scan(uint32_t warp_total, uint32_t* warp_sums, uint32_t& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) warp_sums[warp] = warp_total;
+    __syncthreads();
+    uint32_t v = warp_sums[lane];
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int i = t * E + e;
-        unsigned long long c = ~0ull;
-        if (t < T && i < n && !keep_mask[i]) {
-            uint32_t lab = (uint32_t)label[i];
-            if (lab >= (uint32_t)n) lab = (uint32_t)n - 1;          // out-of-range labels are clamped, never indexed
-            c = ((unsigned long long)lab << 32) | (unsigned long long)i;
-        }
-        r[e] = c;
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += t;
     }
-    block_bitonic_sort<E>(r, comp, T);
+    total = __shfl_sync(0xffffffffu, v, 31);
+    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
+    __syncthreads();
+    return warp == 0 ? 0u : base;
+}
+
+// One walk of a warp over its items with a cursor per (digit, warp) in `cnt`: every item receives the cursor of its
+// digit plus the number of items of the same digit in front of it in its row, and the cursor moves past the row's
+// items.  With the cursors at zero the walk counts (dst null); with the cursors at their scanned values it writes the
+// items to their sorted positions in dst.
+__device__ __forceinline__ void digit_walk(const uint32_t* src, uint32_t* dst, int E, int m, int shift, uint16_t* cnt) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll 1
+    for (int e = 0; e < E; ++e) {
+        const int p = (warp * E + e) * 32 + lane;
+        const bool valid = p < m;
+        const uint32_t item = valid ? src[p] : 0u;
+        const uint32_t d = (item >> shift) & (kDigits - 1);
+        // the lanes of the row that hold the same digit: one ballot per bit
+        const uint32_t vb = __ballot_sync(0xffffffffu, valid);
+        uint32_t peers = valid ? vb : ~vb;
+#pragma unroll
+        for (int k = 0; k < kDigitBits; ++k) {
+            const uint32_t bk = __ballot_sync(0xffffffffu, d >> k & 1u);
+            peers &= (d >> k & 1u) ? bk : ~bk;
+        }
+        const int leader = __ffs(peers) - 1;
+        uint32_t cur = 0;
+        if (valid && lane == leader) {
+            cur = cnt[warp * kCntStride + d];
+            cnt[warp * kCntStride + d] = (uint16_t)(cur + __popc(peers));
+        }
+        cur = __shfl_sync(0xffffffffu, cur, leader);
+        if (dst && valid) dst[cur + __popc(peers & ((1u << lane) - 1u))] = item;
+        __syncwarp();                                      // the next row's leaders may be other lanes
+    }
+}
+
+// Stable sort of m items (label << 16 | token index, in ascending token order on entry) by label: least significant
+// digit first, seven bits at a time, from one buffer to the other and back.  Returns the buffer that holds the result.
+// `cnt`: shared uint16_t [kCntEntries]; label_bits: bits of the largest label.
+__device__ uint32_t* sort_by_label(uint32_t* a, uint32_t* b, int m, int label_bits, uint16_t* cnt, uint32_t* warp_sums) {
+    const int t = threadIdx.x;
+    const int E = (m + kPlanThreads - 1) / kPlanThreads;
+    // this thread's four counters in scan order (digit by digit, inside a digit warp by warp)
+    uint16_t* mine = cnt + (t % (kPlanWarps / 4)) * 4 * kCntStride + t / (kPlanWarps / 4);
+#pragma unroll 1
+    for (int shift = 16; shift < 16 + label_bits; shift += kDigitBits) {
+        for (int c = t; c < kCntEntries; c += kPlanThreads) cnt[c] = 0;
+        __syncthreads();
+        digit_walk(a, nullptr, E, m, shift, cnt);
+        __syncthreads();
+        const uint32_t c0 = mine[0], c1 = mine[kCntStride], c2 = mine[2 * kCntStride], c3 = mine[3 * kCntStride];
+        uint32_t total;
+        const uint32_t b0 = block_exclusive_sum(c0 + c1 + c2 + c3, warp_sums, total);
+        mine[0] = (uint16_t)b0;
+        mine[kCntStride] = (uint16_t)(b0 + c0);
+        mine[2 * kCntStride] = (uint16_t)(b0 + c0 + c1);
+        mine[3 * kCntStride] = (uint16_t)(b0 + c0 + c1 + c2);
+        __syncthreads();
+        digit_walk(a, b, E, m, shift, cnt);
+        __syncthreads();
+        uint32_t* s = a;
+        a = b;
+        b = s;
+    }
+    return a;
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
@@ -46,12 +120,17 @@ merge_plan_kernel(const int32_t* __restrict__ label, const uint8_t* __restrict__
                   const int32_t* __restrict__ vis_len, int vis_len_uniform, int Nv_cap, int Mcap,
                   int32_t* __restrict__ merged_label, int32_t* __restrict__ merged_count,
                   int32_t* __restrict__ n_merged, uint16_t* __restrict__ members, int32_t* __restrict__ starts) {
-    extern __shared__ __align__(16) unsigned long long comp[];   // [P] sorted keys
+    extern __shared__ __align__(16) uint32_t smem_items[];   // two item buffers of Nv_cap (rounded up to 4), then the counters
     __shared__ uint32_t warp_sums[32];
     grid_dependency_wait();
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
     int n = vis_len ? vis_len[b] : vis_len_uniform;
     n = max(0, min(n, Nv_cap));
+    const int cap4 = (Nv_cap + 3) & ~3;
+    uint32_t* buf0 = smem_items;
+    uint32_t* buf1 = smem_items + cap4;
+    uint16_t* cnt = reinterpret_cast<uint16_t*>(smem_items + 2 * cap4);
     label += (size_t)b * Nv_cap;
     keep_mask += (size_t)b * Nv_cap;
     merged_label += (size_t)b * Mcap;
@@ -59,35 +138,79 @@ merge_plan_kernel(const int32_t* __restrict__ label, const uint8_t* __restrict__
     members += (size_t)b * Nv_cap;
     starts += (size_t)b * Mcap;
 
-    int P = 256;                                          // at least one warp of 8 keys per thread
-    while (P < n) P <<= 1;
-    if (P <= 8 * kPlanThreads) sort_members<8>(label, keep_mask, n, P / 8, comp);
-    else sort_members<16>(label, keep_mask, n, P / 16, comp);
-
-    // run heads -> merged rows (ascending label); run tails close them; the sorted indices are the member list
-    uint32_t heads = 0, tails = 0;
-    for (int base = 0; base < P; base += kPlanThreads) {
-        const int p = base + tid;
-        const unsigned long long c = p < n ? comp[p] : ~0ull;     // non-elite tokens sort to the front, at most n of them
-        const bool valid = c != ~0ull;
-        const uint32_t lab = (uint32_t)(c >> 32);
-        const bool head = valid && (p == 0 || (uint32_t)(comp[p - 1] >> 32) != lab);
-        const bool tail = valid && (p + 1 >= n || comp[p + 1] == ~0ull || (uint32_t)(comp[p + 1] >> 32) != lab);
-        if (valid) members[p] = (uint16_t)(c & 0xFFFFull);
-        uint32_t th, tt;
-        const uint32_t hs = heads + block_prefix_count(head, warp_sums, th);
-        const uint32_t ts = tails + block_prefix_count(tail, warp_sums, tt);
-        if (head && hs < (uint32_t)Mcap) {
-            merged_label[hs] = (int32_t)lab;
-            starts[hs] = p;
+    // ---- the non-elite tokens, in token order: count per warp, one scan, then place.  (Unrolled, unlike the walks
+    //      over shared memory: all of a thread's global loads are in flight together.)
+    uint32_t m;
+    {
+        const int E = (n + kPlanThreads - 1) / kPlanThreads;
+        uint32_t it[kPlanItems], take = 0, mine = 0;
+#pragma unroll
+        for (int e = 0; e < kPlanItems; ++e) {
+            const int i = (warp * E + e) * 32 + lane;
+            if (e < E && i < n) {
+                uint32_t lab = (uint32_t)label[i];
+                if (lab >= (uint32_t)n) lab = (uint32_t)n - 1;     // out-of-range labels are clamped, never indexed
+                it[e] = (lab << 16) | (uint32_t)i;
+                if (!keep_mask[i]) take |= 1u << e;
+            }
         }
-        if (tail && ts < (uint32_t)Mcap) merged_count[ts] = p;          // position of the run's last member for now
-        heads += th;
-        tails += tt;
-        if (base + kPlanThreads >= n) break;                            // uniform
+#pragma unroll
+        for (int e = 0; e < kPlanItems; ++e) mine += __popc(__ballot_sync(0xffffffffu, take >> e & 1u));
+        uint32_t pos = warp_totals_scan(mine, warp_sums, m);
+#pragma unroll
+        for (int e = 0; e < kPlanItems; ++e) {
+            const uint32_t bal = __ballot_sync(0xffffffffu, take >> e & 1u);
+            if (take >> e & 1u) buf0[pos + __popc(bal & lt)] = it[e];
+            pos += __popc(bal);
+        }
     }
     __syncthreads();
-    for (int m = tid; m < min((int)heads, Mcap); m += kPlanThreads) merged_count[m] = merged_count[m] - starts[m] + 1;
+    // ---- members of a cluster side by side, in ascending token order; clusters in ascending label order
+    const uint32_t* items = sort_by_label(buf0, buf1, (int)m, n > 1 ? 32 - __clz(n - 1) : 0, cnt, warp_sums);
+
+    // ---- run heads -> merged rows; run tails close them; the sorted indices are the member list
+    const int E = ((int)m + kPlanThreads - 1) / kPlanThreads;
+    uint32_t wh = 0, wt = 0;
+#pragma unroll 1
+    for (int e = 0; e < E; ++e) {
+        const int p = (warp * E + e) * 32 + lane;
+        bool head = false, tail = false;
+        if (p < (int)m) {
+            const uint32_t c = items[p], lab = c >> 16;
+            head = p == 0 || (items[p - 1] >> 16) != lab;
+            tail = p + 1 >= (int)m || (items[p + 1] >> 16) != lab;
+            members[p] = (uint16_t)(c & 0xFFFFu);
+        }
+        wh += __popc(__ballot_sync(0xffffffffu, head));
+        wt += __popc(__ballot_sync(0xffffffffu, tail));
+    }
+    // (two 16-bit counts in a word: neither can exceed 16384)
+    uint32_t totals;
+    const uint32_t before = warp_totals_scan(wh | (wt << 16), warp_sums, totals);
+    uint32_t hs = before & 0xFFFFu, ts = before >> 16;
+    const uint32_t heads = totals & 0xFFFFu;
+#pragma unroll 1
+    for (int e = 0; e < E; ++e) {
+        const int p = (warp * E + e) * 32 + lane;
+        bool head = false, tail = false;
+        uint32_t lab = 0;
+        if (p < (int)m) {
+            lab = items[p] >> 16;
+            head = p == 0 || (items[p - 1] >> 16) != lab;
+            tail = p + 1 >= (int)m || (items[p + 1] >> 16) != lab;
+        }
+        const uint32_t hb = __ballot_sync(0xffffffffu, head), tb = __ballot_sync(0xffffffffu, tail);
+        const uint32_t h = hs + __popc(hb & lt), t = ts + __popc(tb & lt);
+        if (head && h < (uint32_t)Mcap) {
+            merged_label[h] = (int32_t)lab;
+            starts[h] = p;
+        }
+        if (tail && t < (uint32_t)Mcap) merged_count[t] = p;            // position of the run's last member for now
+        hs += __popc(hb);
+        ts += __popc(tb);
+    }
+    __syncthreads();
+    for (int mm = tid; mm < min((int)heads, Mcap); mm += kPlanThreads) merged_count[mm] = merged_count[mm] - starts[mm] + 1;
     if (tid == 0) n_merged[b] = (int32_t)heads;
     grid_dependency_launch_dependents();
 }
@@ -136,16 +259,19 @@ merge_rows_kernel(const uint4* __restrict__ hidden, int N, int dh8, int vis_star
 #pragma unroll
     for (int u = 0; u < 8; ++u) partial[g][lane][u] = acc[u];
     __syncthreads();
-    const int pl = tid & 31, k = tid >> 5;                // this thread finishes element k of piece pl
+    const int pl = tid & 31;                              // this thread finishes elements tid / 32, + G, .. of piece pl
     const int pcol = blockIdx.z * 32 + pl;
     if (pcol >= dh8) return;
-    float sum = 0.f;
 #pragma unroll
-    for (int q = 0; q < G; ++q) sum += partial[q][pl][k];   // warp order: fixed
-    sum = sum / (float)count;
-    const size_t o = (((size_t)b * Mcap + m) * dh8 + pcol) * 8 + k;
-    if (merged_f32) merged_f32[o] = sum;
-    if (merged_bf16) static_cast<__nv_bfloat16*>(merged_bf16)[o] = __float2bfloat16_rn(sum);
+    for (int k = tid >> 5; k < 8; k += G) {
+        float sum = 0.f;
+#pragma unroll
+        for (int q = 0; q < G; ++q) sum += partial[q][pl][k];   // warp order: fixed
+        sum = sum / (float)count;
+        const size_t o = (((size_t)b * Mcap + m) * dh8 + pcol) * 8 + k;
+        if (merged_f32) merged_f32[o] = sum;
+        if (merged_bf16) static_cast<__nv_bfloat16*>(merged_bf16)[o] = __float2bfloat16_rn(sum);
+    }
 }
 
 // Workspace: status | members uint16 [B, Nv_cap] | starts int32 [B, Mcap]
@@ -176,9 +302,7 @@ int launch_merge(const void* hidden, int B, int N, int Dh, int vis_start, const 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     {
-        int P = 256;
-        while (P < Nv_cap) P <<= 1;
-        const size_t smem = (size_t)P * sizeof(unsigned long long);
+        const size_t smem = 2 * (size_t)((Nv_cap + 3) & ~3) * sizeof(uint32_t) + (size_t)kCntEntries * sizeof(uint16_t);
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(merge_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return record_cuda(e);
