@@ -285,7 +285,7 @@ int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh,
  *   q_cls     bf16 [B, H, d]      query of the [CLS] token per head (d multiple of 8)
  *   K         bf16 [B, H, M, d]   keys of the layer; key 0 belongs to [CLS]
  *   scale     usually 1 / sqrt(d)
- *   saliency  fp32 [B, M - 1] out: S of the visual tokens 1 .. M-1
+ *   saliency  fp32 [B, M - 1] out: S of the visual tokens 1 .. M-1 (may be NULL when M <= 1: nothing to write)
  *   cls_self  fp32 [B] out, optional: attention of [CLS] to itself, summed over heads
  *   workspace vitcop_workspace_bytes(VITCOP_OP_SALIENCY, B, H, M, ...) bytes
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */

@@ -404,7 +404,7 @@ int vitcop_merge_clusters(const void* hidden, int B, int N, int Dh, int vis_star
 
 int vitcop_cls_saliency(const void* q_cls, const void* K, int B, int H, int M, int d, float scale, float* saliency,
                         float* cls_self, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!q_cls || !K || !saliency || B < 0 || H < 0 || M < 0 || d < 0) return VITCOP_ERR_INVALID_ARG;
+    if (!q_cls || !K || (!saliency && M > 1) || B < 0 || H < 0 || M < 0 || d < 0) return VITCOP_ERR_INVALID_ARG;
     if (d % 8 || !aligned16(q_cls) || !aligned16(K) || B > 65535 || H > 4096 || d > 4096) return VITCOP_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < saliency_workspace_bytes(B, H, M) || !aligned256(workspace))
         return VITCOP_ERR_WORKSPACE;

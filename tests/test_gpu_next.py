@@ -73,6 +73,38 @@ def test_merge_small_and_edges():
     _check_merge(hid, 0, 700, np.zeros((1, 700), np.int32), (rng.random((1, 700)) < 0.1).astype(np.uint8), 4)
 
 
+@pytest.mark.parametrize("n,clusters,keep_p", [(16384, 820, 0.06), (16384, 16384, 0.5), (9000, 3, 0.0), (1025, 1025, 0.2),
+                                               (31, 5, 0.3), (1, 1, 0.0)])
+def test_merge_planner_sizes(n, clusters, keep_p):
+    """The planner at the largest span, with every token its own cluster, with a few huge clusters, and at sizes around
+    its row (32) and pass (1024) granularity; labels are arbitrary token indices, one of them out of range."""
+    rng = np.random.default_rng(n + clusters)
+    B, Dh, vs = 2, 64, 3
+    hid = W.f32_to_bf16_bits(rng.standard_normal((B, n + vs + 2, Dh)).astype(np.float32))
+    ids = np.sort(rng.choice(n, size=clusters, replace=False)).astype(np.int32)
+    label = ids[rng.integers(0, clusters, size=(B, n))]
+    keep = (rng.random((B, n)) < keep_p).astype(np.uint8)
+    vl = np.array([n, max(0, n - 7)], dtype=np.int32)
+    label[1, : vl[1]] = np.minimum(label[1, : vl[1]], max(vl[1] - 1, 0))      # labels stay inside the sample's own span
+    _check_merge(hid, vs, vl, label, keep, min(n, 900))
+
+
+def test_merge_label_out_of_range_is_clamped():
+    rng = np.random.default_rng(11)
+    n, Dh = 100, 64
+    hid = W.f32_to_bf16_bits(rng.standard_normal((1, n, Dh)).astype(np.float32))
+    label = rng.integers(0, 7, size=(1, n)).astype(np.int32)
+    bad = label.copy()
+    bad[0, 5], bad[0, 50] = 10 ** 6, -3
+    ref = label.copy()
+    ref[0, 5] = ref[0, 50] = n - 1
+    keep = np.zeros((1, n), np.uint8)
+    a = _gpu_merge(hid, 0, n, bad, keep, n)
+    b = _gpu_merge(hid, 0, n, ref, keep, n)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
 @pytest.mark.parametrize("name", ["tiny", "c0"])
 def test_stage_two_with_merge(name):
     """Stage II as Algorithm 3 states it: VIC labels -> K-norm quota elites -> merged token per cluster."""
@@ -93,7 +125,11 @@ def test_stage_two_with_merge(name):
         assert mc[b, :nm[b]].sum() == w.Nv - nk[b]
 
 
-@pytest.mark.parametrize("B,H,M,d", [(2, 4, 33, 16), (1, 1, 2, 8), (3, 16, 577, 64), (2, 12, 1300, 128)])
+# shapes: a row on 8 / 16 / 32 lanes (d up to 64 / 128 / 256), rows longer than 32 pieces (d = 264, 512), one key
+# only, more heads than the second kernel has warps, key counts around the chunk (256) and block (64) sizes
+@pytest.mark.parametrize("B,H,M,d", [(2, 4, 33, 16), (1, 1, 2, 8), (3, 16, 577, 64), (2, 12, 1300, 128),
+                                     (2, 3, 300, 256), (1, 2, 70, 264), (1, 2, 257, 512), (2, 5, 1, 64),
+                                     (1, 19, 256, 72), (1, 40, 65, 32), (1, 2, 4100, 128)])
 def test_cls_saliency(B, H, M, d):
     q, K = W.make_cls_qk(M, B, H, M, d)
     scale = 1.0 / np.sqrt(d)
@@ -105,6 +141,7 @@ def test_cls_saliency(B, H, M, d):
     S, c = S.cpu().numpy(), c.cpu().numpy()
     for b in range(B):
         want, wc = oracle.cls_saliency(q[b], K[b], scale)
+        assert S[b].shape == want.shape
         assert np.all(rel_err(S[b], want) <= SAL_RTOL) and abs(c[b] - wc) <= SAL_RTOL * wc
         assert abs(S[b].sum() + c[b] - H) <= 1e-4             # every head's attention row sums to one
 
