@@ -23,17 +23,46 @@ namespace {
 // ------------------------------------------------------------------------------------------------
 // small kernels
 // ------------------------------------------------------------------------------------------------
-// rho[b,i] = sum of the partials of the tiles that hold token i, in a fixed order (reproducible bits):
-// the row-side slots of the column tiles that pair row tile i / 128 with later tokens, then the column-side
-// slots of the row tiles that pair column tile i / BN with earlier tokens.
+// rho[b,i] = sum of the partials of the tiles that hold token i, in a fixed order (reproducible bits): the row-side
+// slots of the column tiles that pair row tile i / 128 with later tokens, then the column-side slots of the row tiles
+// that pair column tile i / BN with earlier tokens -- one contiguous range of slots.  LANES neighbouring lanes share a
+// token: each adds its part of the range slot by slot (sixteen independent loads at a time), and the sums are added
+// in lane order.  A long sample has up to 190 slots per token, which one thread alone would fetch in a dozen
+// dependent rounds; for a few dozen slots one thread per token is the faster shape.
+constexpr int kRhoLanesLong = 4;
+constexpr int kRhoLongSlots = 64;                          // samples with more slots than this take kRhoLanesLong lanes
+template <int LANES>
 __global__ void rho_reduce_kernel(const float* __restrict__ part, int n, GramTiling t, float* __restrict__ rho,
                                   float* __restrict__ rho_user) {
     grid_dependency_launch_dependents();
     grid_dependency_wait();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int q = threadIdx.x % LANES;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) / LANES;
     const int b = blockIdx.y;
-    if (i >= n) return;
-    const float s = rho_from_partials(part + (size_t)b * t.slots() * t.n_pad + i, t, i);
+    const bool valid = i < n;                              // (all lanes stay for the shuffles)
+    float s = 0.f;
+    if (valid) {
+        const int ti = i / kGramBM, tj = i / t.BN;
+        const int cap = t.R * (tj + 1);
+        const int first = ti / t.R, last = t.TJ + (t.TI < cap ? t.TI : cap);
+        const int per = (last - first + LANES - 1) / LANES;
+        const int c0 = first + q * per, c1 = min(last, c0 + per);
+        const float* p = part + (size_t)b * t.slots() * t.n_pad + i;
+        for (int c = c0; c < c1; c += 16) {
+            float v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) v[u] = (c + u < c1) ? p[(size_t)(c + u) * t.n_pad] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                if (c + u < c1) s += v[u];
+        }
+    }
+    float others[LANES];
+#pragma unroll
+    for (int u = 1; u < LANES; ++u) others[u] = __shfl_down_sync(0xffffffffu, s, u);
+    if (!valid || q != 0) return;
+#pragma unroll
+    for (int u = 1; u < LANES; ++u) s += others[u];
     rho[(size_t)b * n + i] = s;
     if (rho_user) rho_user[(size_t)b * n + i] = s;
 }
@@ -386,9 +415,11 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
         {
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attr[1];
-            pdl_config(cfg, attr, dim3((n + 255) / 256, B), dim3(256), 0, stream, true);
+            const int lanes = tiling.slots() > kRhoLongSlots ? kRhoLanesLong : 1;
+            pdl_config(cfg, attr, dim3((n * lanes + 255) / 256, B), dim3(256), 0, stream, true);
             KernelTimeScope timed("rho_reduce_kernel", stream);
-            rc = record_cuda(cudaLaunchKernelEx(&cfg, rho_reduce_kernel, (const float*)part, n, tiling, rho, rho_user));
+            rc = record_cuda(cudaLaunchKernelEx(&cfg, lanes == 1 ? rho_reduce_kernel<1> : rho_reduce_kernel<kRhoLanesLong>,
+                                                (const float*)part, n, tiling, rho, rho_user));
             if (rc != VITCOP_OK) return rc;
         }
         if (!keep_tiles) {
