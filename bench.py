@@ -323,6 +323,27 @@ def pinned_inputs(w, torch):
     return out
 
 
+def tiles_within_radius(w):
+    """Share of the 128 x 256 tiles of the symmetric half whose row block and column blocks lie within the spatial radius
+    of one another (bounding boxes of the blocks' positions, fp32): the tiles the density sweep keeps and the delta pass
+    reads.  Computed here from the positions alone."""
+    pos = W.make_positions(w).astype(np.float32)
+    n, tau2 = w.Nv, np.float32(w.tau) ** 2
+    TI, TJ = -(-n // 128), -(-n // 256)
+    kept = total = 0
+    for b in range(pos.shape[0]):
+        lo = np.stack([pos[b, i * 128:(i + 1) * 128].min(0) for i in range(TI)])
+        hi = np.stack([pos[b, i * 128:(i + 1) * 128].max(0) for i in range(TI)])
+        for tj in range(TJ):
+            cl, ch = lo[2 * tj:2 * tj + 2].min(0), hi[2 * tj:2 * tj + 2].max(0)
+            rows = min(TI, 2 * tj + 2)
+            d = np.maximum(np.float32(0), np.maximum(lo[:rows] - ch, cl - hi[:rows]))
+            s2 = d[:, 0] * d[:, 0] + d[:, 1] * d[:, 1]
+            kept += int(np.count_nonzero(~(s2 > tau2)))
+            total += rows
+    return kept / max(total, 1)
+
+
 def algorithmic_units(w, s, vis_in, kept):
     """Per launch at step s: kernel -> (bound, algorithmic bytes or flop).
 
@@ -338,8 +359,10 @@ def algorithmic_units(w, s, vis_in, kept):
         sweep = w.B * w.Nv * (w.Nv + 1) * w.D
         u.update({"gram_resident_kernel": ("tensor", sweep), "gram_tc_kernel<rho>": ("tensor", sweep),
                   "gram_tc_kernel<delta>": ("tensor", sweep),
-                  # reads the stored Gram value of every pair of the symmetric half (diagonal included) once: 4 bytes
-                  "delta_pass_kernel": ("hbm", w.B * w.Nv * (w.Nv + 1) // 2 * 4)})
+                  # reads the stored Gram value of every pair of the symmetric half (diagonal included) that sits in
+                  # a tile within the spatial radius, once: 4 bytes
+                  "delta_pass_kernel": ("hbm", int(w.B * w.Nv * (w.Nv + 1) // 2 * 4 * tiles_within_radius(w))
+                                        if w.Nv >= 8192 else 0)})
     return u
 
 

@@ -73,34 +73,49 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
     const int quarter = warp & 3, slice = warp >> 2;
     const int rl = quarter * 32 + lane;                    // tile-local row of this thread
 
-    const long long t_begin = total_tiles * blockIdx.x / gridDim.x, t_end = total_tiles * (blockIdx.x + 1) / gridDim.x;
-    // The tiles of the run are contiguous in memory, so the thread's loads form one stream over the whole run: the
-    // sixteen columns it works on (A, B: eight each) and the sixteen after those, requested while it works -- across
-    // tile boundaries, so that the constants of a new tile are fetched with data already in flight.  `pf` walks that
-    // stream: two float4 columns of 128 rows per group, and past the other half's columns at the end of a tile.
+    // Tiles whose row block lies beyond the spatial radius of their column blocks were not kept by the density sweep
+    // and are not read here: g.kept lists the numbers of the others in ascending order (filter.cu), and the CTAs
+    // share that list out evenly.  Without a radius every tile is kept and the list is the identity.
+    const long long n_list = g.kept ? (long long)*g.n_kept : total_tiles;
+    const long long k_begin = n_list * blockIdx.x / gridDim.x;
+    const int run = (int)(n_list * (blockIdx.x + 1) / gridDim.x - k_begin);     // this CTA's entries: k_begin + [0, run)
+    if (run <= 0) return;                                  // (uniform)
+    const int32_t* const kept = g.kept ? g.kept + k_begin : nullptr;
+    auto tile_of = [&](int k) { return kept ? (long long)kept[k] : k_begin + k; };
+    __shared__ long long s_next;                           // number of the tile after the current one (-1: none)
+    int k = 0;
+    long long t = tile_of(0);
+    // The thread's loads form one stream over the tiles of the run: the sixteen columns it works on (A, B: eight
+    // each) and the sixteen after those, requested while it works -- across tile boundaries, so that the constants of
+    // a new tile are fetched with data already in flight.  `pf` walks that stream: two float4 columns of 128 rows per
+    // group; after a tile's last group it moves on to the next tile that is kept (s_next; null after the last).
     constexpr size_t kGroupStep = 2 * BM;                                      // float4 per group
-    constexpr size_t kTileSkip = gram_tile_floats(BN) / 4 - (size_t)kGroups * kGroupStep;
-    const float4* pf = reinterpret_cast<const float4*>(g.gram_tiles) + (size_t)t_begin * (gram_tile_floats(BN) / 4) +
-                       (size_t)(slice * kSliceCols / 4) * BM + rl;
-    const float4* const pf_end = reinterpret_cast<const float4*>(g.gram_tiles) + (size_t)t_end * (gram_tile_floats(BN) / 4);
+    const float4* const tiles0 = reinterpret_cast<const float4*>(g.gram_tiles) + (size_t)(slice * kSliceCols / 4) * BM + rl;
+    auto tile_ptr = [&](long long tt) { return tiles0 + (size_t)tt * (gram_tile_floats(BN) / 4); };
+    const float4* pf = tile_ptr(t);
     float4 A0 = make_float4(0.f, 0.f, 0.f, 0.f), A1 = A0, B0 = A0, B1 = A0;
     int pf_group = 0;                                      // group inside its tile that pf points at
     auto fetch_pair = [&](float4& x0, float4& x1, float4& y0, float4& y1) {    // the next two groups of the stream
-        if (pf < pf_end) {
+        if (pf) {
             x0 = ld_tile(pf);
             x1 = ld_tile(pf + BM);
             y0 = ld_tile(pf + kGroupStep);
             y1 = ld_tile(pf + kGroupStep + BM);
+            pf += 2 * kGroupStep;
         }
-        pf += 2 * kGroupStep;
         pf_group += 2;
-        if (pf_group == kGroups) { pf_group = 0; pf += kTileSkip; }
+        if (pf_group == kGroups) {
+            pf_group = 0;
+            const long long tn = s_next;
+            pf = tn >= 0 ? tile_ptr(tn) : nullptr;
+        }
     };
     fetch_pair(A0, A1, B0, B1);
     int prev_b = -1, prev_tj = -1;
-    for (long long t = t_begin; t < t_end; ++t) {
+    for (; k < run; ++k) {
         int b, ti, tj;
         decode_sym_tile(tl, t, b, ti, tj);
+        if (threadIdx.x == 0) s_next = k + 1 < run ? tile_of(k + 1) : -1;   // (published by the barrier behind the tile's constants)
         const bool same_cols = b == prev_b && tj == prev_tj;       // the column block of the previous tile: its constants stay
         prev_b = b;
         prev_tj = tj;
@@ -235,6 +250,7 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
             A0 = N0; A1 = N1; B0 = M0; B1 = M1;
         }
 
+        const long long t_next = s_next;                   // (rewritten only behind the barriers below)
         // ---- combine the four column slices of every row and the four row quarters of every column
         if (slice > 0) {
             rowred[(slice - 1) * BM + rl] = rbest;
@@ -256,6 +272,7 @@ delta_pass_kernel(const GramArgs g, const GramTiling tl, const long long total_t
             if (cb != ~0ull && J0 + ce < g.n) atomicMin(g.best + bo + J0 + ce, cb);
         }
         __syncthreads();                                   // the shared arrays are rewritten for the next tile
+        t = t_next;
     }
 }
 

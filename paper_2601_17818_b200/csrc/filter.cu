@@ -67,6 +67,59 @@ __global__ void rho_reduce_kernel(const float* __restrict__ part, int n, GramTil
     if (rho_user) rho_user[(size_t)b * n + i] = s;
 }
 
+// The tiles of the symmetric numbering that lie within the spatial radius (gram.cuh: tile_outside_radius), in
+// ascending order: list[0 .. *count).  One small CTA that fits on an SM beside a CTA of the density sweep: it is
+// queued behind that sweep, does its work while the sweep runs and only then waits for it, so that the kernels
+// queued behind see both complete.  Thread t tests the tiles [t E, (t + 1) E) of a round of 256 E tiles with all its
+// loads in flight; one scan per round places them.
+constexpr int kKeptThreads = 256;
+constexpr int kKeptPerThread = 16;
+__global__ void __launch_bounds__(kKeptThreads)
+kept_tiles_kernel(const float4* __restrict__ bbox, GramTiling t, long long total, float tau2, int32_t* __restrict__ list,
+                  int32_t* __restrict__ count) {
+    __shared__ uint32_t warp_sums[kKeptThreads / 32];
+    grid_dependency_launch_dependents();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t placed = 0;
+    for (long long base = 0; base < total; base += (long long)kKeptThreads * kKeptPerThread) {
+        uint32_t keep = 0;
+#pragma unroll
+        for (int e = 0; e < kKeptPerThread; ++e) {
+            const long long tile = base + (long long)threadIdx.x * kKeptPerThread + e;
+            if (tile < total) {
+                int b, ti, tj;
+                decode_sym_tile(t, tile, b, ti, tj);
+                if (!tile_outside_radius(bbox + (size_t)b * t.TI, t, ti, tj, tau2)) keep |= 1u << e;
+            }
+        }
+        // exclusive prefix of the per-thread counts over the CTA, in thread order
+        const uint32_t mine = __popc(keep);
+        uint32_t incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        __syncthreads();                                   // (the previous round's sums have been read)
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        uint32_t before = 0, round_total = 0;
+#pragma unroll
+        for (int w = 0; w < kKeptThreads / 32; ++w) {
+            const uint32_t v = warp_sums[w];
+            if (w < warp) before += v;
+            round_total += v;
+        }
+        uint32_t pos = placed + before + incl - mine;
+#pragma unroll
+        for (int e = 0; e < kKeptPerThread; ++e)
+            if (keep >> e & 1u) list[pos++] = (int32_t)(base + (long long)threadIdx.x * kKeptPerThread + e);
+        placed += round_total;
+    }
+    if (threadIdx.x == 0) *count = (int32_t)placed;
+    grid_dependency_wait();
+}
+
 // ------------------------------------------------------------------------------------------------
 // Centres, forest roots and labels: one CTA per sample.
 // ------------------------------------------------------------------------------------------------
@@ -314,11 +367,12 @@ vic_finalize_kernel(const uint16_t* __restrict__ feat, int n, int D, int n_cente
 // host side
 // ------------------------------------------------------------------------------------------------
 // Workspace of the filter: status block | row-block flags [B, ceil(n / 128)] | w | a | rho | best |
-// rho partials [B, slots, n_pad] (sized for either tile width) | Gram tiles of the density sweep (problems too large
+// rho partials [B, slots, n_pad] (sized for either tile width) | bounding boxes of the row blocks' positions |
+// count and list of the tiles within the spatial radius | Gram tiles of the density sweep (problems too large
 // for the one-kernel sweep: 4 bytes per pair of the symmetric half, tile padding included).  The status block and the
 // flags are zeroed at the start of every call.  Words of the status block: 0 status, 2 grid barrier.
 struct FilterWs {
-    size_t off_flags, off_w, off_a, off_rho, off_best, off_part, off_tiles, total;
+    size_t off_flags, off_w, off_a, off_rho, off_best, off_part, off_bbox, off_kept, off_tiles, total;
     FilterWs(int B, int n) {
         size_t o = kStatusBytes;
         const size_t bn = (size_t)B * n;
@@ -329,10 +383,14 @@ struct FilterWs {
         off_best = o; o += align_up(bn * 8, 256);
         const GramTiling t = make_gram_tiling(n, 128);           // the narrow tiling has the most slots
         off_part = o; o += align_up((size_t)B * t.slots() * t.n_pad * 4, 256);
-        off_tiles = o;
+        off_bbox = o;   o += align_up((size_t)B * t.TI * sizeof(float4), 256);
+        off_kept = off_tiles = o;
         if (gram_keeps_tiles(B, n)) {
             const int bn = gram_pick_bn(B, n);
-            o += align_up((size_t)B * make_gram_tiling(n, bn).tiles_per_b * gram_tile_floats(bn) * 4, 256);
+            const size_t tiles = (size_t)B * make_gram_tiling(n, bn).tiles_per_b;
+            o += align_up((tiles + 1) * sizeof(int32_t), 256);    // count, then the list of kept tiles
+            off_tiles = o;
+            o += align_up(tiles * gram_tile_floats(bn) * 4, 256);
         }
         total = o;
     }
@@ -408,10 +466,28 @@ int launch_filter(const void* feat, const float* pos, int B, int n, int D, const
     } else {
         const bool keep_tiles = gram_keeps_tiles(B, n);
         g.gram_tiles = keep_tiles ? reinterpret_cast<float*>(ws + l.off_tiles) : nullptr;
+        // with a spatial radius, tiles beyond it are neither kept nor read back (gram.cuh: tile_outside_radius)
+        g.bbox = (keep_tiles && g.tau2 >= 0.f) ? reinterpret_cast<float4*>(ws + l.off_bbox) : nullptr;
         rc = launch_gram_sweep(GRAM_DIAG, feat, g, make_gram_tiling(n, 128), stream, false);
         if (rc != VITCOP_OK) return rc;
         rc = launch_gram_sweep(GRAM_RHO, feat, g, tiling, stream, true);
         if (rc != VITCOP_OK) return rc;
+        if (g.bbox) {
+            // which tiles the delta pass will read: one small CTA beside the density sweep (the boxes come from the
+            // diagonal sweep, complete since the density sweep's epilogues started)
+            int32_t* cnt = reinterpret_cast<int32_t*>(ws + l.off_kept);
+            const long long tiles = (long long)B * tiling.tiles_per_b;
+            if (tiles > 0x7fffffffLL) return VITCOP_ERR_UNSUPPORTED;
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[1];
+            pdl_config(cfg, attr, dim3(1), dim3(kKeptThreads), 0, stream, true);
+            KernelTimeScope timed("kept_tiles_kernel", stream);
+            rc = record_cuda(cudaLaunchKernelEx(&cfg, kept_tiles_kernel, (const float4*)g.bbox, tiling, tiles, g.tau2, cnt + 1,
+                                                cnt));
+            if (rc != VITCOP_OK) return rc;
+            g.kept = cnt + 1;
+            g.n_kept = cnt;
+        }
         {
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attr[1];

@@ -495,6 +495,35 @@ __device__ __forceinline__ bool epi_tile(const KernelArgs& k, const EpiSmem& sm,
         }
     }
 
+    if (MODE == GRAM_DIAG && g.bbox) {
+        // ---- bounding box of the row block's positions: per warp by shuffles, the four row quarters through shared
+        //      memory (rows outside the sample and coordinates that are not numbers leave the box alone)
+        if (slice == 0) {
+            float4 bx = make_float4(kInf, kInf, -kInf, -kInf);
+            if (row_valid) {
+                const float2 q = *reinterpret_cast<const float2*>(g.pos + 2 * (bo + i));
+                bx = make_float4(q.x, q.y, q.x, q.y);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                bx.x = fminf(bx.x, __shfl_xor_sync(0xffffffffu, bx.x, off));
+                bx.y = fminf(bx.y, __shfl_xor_sync(0xffffffffu, bx.y, off));
+                bx.z = fmaxf(bx.z, __shfl_xor_sync(0xffffffffu, bx.z, off));
+                bx.w = fmaxf(bx.w, __shfl_xor_sync(0xffffffffu, bx.w, off));
+            }
+            if (lane == 0) reinterpret_cast<float4*>(rowred)[quarter] = bx;
+        }
+        epi_bar_sync<kEpiThreads>();
+        if (e == 0 && ok) {
+            float4 bx = reinterpret_cast<const float4*>(rowred)[0];
+#pragma unroll
+            for (int q = 1; q < 4; ++q) {
+                const float4 o = reinterpret_cast<const float4*>(rowred)[q];
+                bx = make_float4(fminf(bx.x, o.x), fminf(bx.y, o.y), fmaxf(bx.z, o.z), fmaxf(bx.w, o.w));
+            }
+            g.bbox[(size_t)b * k.t.TI + ti] = bx;
+        }
+    }
     if (SYM) {
         // ---- combine the four column slices of every row and the four row quarters of every column
         if (slice > 0) {
@@ -578,6 +607,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t bar_drain = bar_tempty + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S::kStages + 5);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // (the last words of the barrier block hold the epilogue's mask of tiles that are not kept)
+    static_assert((2 * S::kStages + 5) * 8 + 8 + (NS * 128 / 32) * 4 <= S::kBarBytes, "barrier block too small");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr uint32_t kTmemCols = 2 * BN;
@@ -603,9 +634,12 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // The kernels that follow on the stream may be scheduled from here on; they wait for this grid to
-    // complete before they touch anything it writes.
-    grid_dependency_launch_dependents();
+    // The kernels that follow on the stream may be scheduled from here on; they wait for this grid to complete
+    // before they touch anything it writes.  A density sweep that has a kernel running beside it (filter.cu: the list
+    // of tiles within the spatial radius) releases them only once its own predecessors are complete, so that the
+    // neighbour may rely on their results without a wait of its own.
+    const bool release_late = MODE == GRAM_RHO && g.bbox != nullptr;
+    if (!release_late) grid_dependency_launch_dependents();
 
     const long long total_tiles = k.total_tiles;
     const int KB = g.D / BK;
@@ -675,8 +709,12 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ epilogue (warps 2 ..)
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
+        const bool skip_far = MODE == GRAM_RHO && g.gram_tiles && g.bbox;
+        uint32_t* far_mask = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + S::kBarBytes) - kEpiThreads / 32;
+        long long kt = 0;                                  // tiles this CTA has taken
 
         grid_dependency_wait();                            // w, a, rho, best come from the preceding kernels
+        if (release_late) grid_dependency_launch_dependents();
 
         for (long long t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             EpiCall c;
@@ -689,6 +727,26 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             c.abort_flag = abort_flag;
             c.limit_ns = k.limit_of(kRoleEpi);
             c.store = (MODE == GRAM_RHO && g.gram_tiles) ? g.gram_tiles + (size_t)t * gram_tile_floats(BN) : nullptr;
+            if (skip_far) {
+                // a tile beyond the spatial radius is of no use to Eq. 3 and is not kept (gram.cuh:
+                // tile_outside_radius); the CTA's next kEpiThreads tiles are tested together, one per thread
+                const int kk = (int)(kt % kEpiThreads);
+                if (kk == 0) {
+                    epi_bar_sync<kEpiThreads>();               // (the previous mask has been read by everyone)
+                    const long long mine = t + (long long)(threadIdx.x - 64) * gridDim.x;
+                    bool far = false;
+                    if (mine < total_tiles) {
+                        int fb, fti, ftj;
+                        decode_tile<BN, SYM, DIAG>(k, mine, fb, fti, ftj);
+                        far = tile_outside_radius(g.bbox + (size_t)fb * k.t.TI, k.t, fti, ftj, g.tau2);
+                    }
+                    const uint32_t bal = __ballot_sync(0xffffffffu, far);
+                    if (lane == 0) far_mask[warp - 2] = bal;
+                    epi_bar_sync<kEpiThreads>();
+                }
+                if (far_mask[kk >> 5] >> (kk & 31) & 1u) c.store = nullptr;
+            }
+            ++kt;
             if (epi_tile<BN, MODE, METRIC, SPATIAL, NS>(k, sm, c, ok)) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }

@@ -102,8 +102,31 @@ struct GramArgs {
     const void* kn_K;
     float* kn_score;
     int kn_B, kn_H, kn_N, kn_d, kn_vis_start, kn_Nv;
+    float4* bbox;               // [B, ceil(n / 128)] bounding box (min x, min y, max x, max y) of every row block's
+                                // positions, or nullptr: written by GRAM_DIAG, read where whole tiles are skipped
+    const int32_t* kept;        // delta pass, optional: numbers of the tiles to read, ascending; nullptr = all of them
+    const int32_t* n_kept;      // their count (device)
     int* status;                // device status word
 };
+
+// Eq. 3 only pairs tokens within the spatial radius, so a tile whose row block lies farther than the radius from its
+// column blocks cannot contribute: the density sweep need not keep it and the delta pass need not read it.  The
+// distance between the bounding boxes is taken with the operations of the per-pair test (fp32 differences, squares
+// joined by one fma), all of them monotone, so it never exceeds the distance of any pair of the tile: what is
+// skipped is exactly what the per-pair test would have rejected.  `bbox_b`: the sample's boxes.
+__device__ __forceinline__ bool tile_outside_radius(const float4* __restrict__ bbox_b, const GramTiling& t, int ti, int tj,
+                                                    float tau2) {
+    const float4 r = bbox_b[ti];
+    float4 c = bbox_b[t.R * tj];
+    for (int k = 1; k < t.R; ++k) {
+        if (t.R * tj + k >= t.TI) break;
+        const float4 o = bbox_b[t.R * tj + k];
+        c = make_float4(fminf(c.x, o.x), fminf(c.y, o.y), fmaxf(c.z, o.z), fmaxf(c.w, o.w));
+    }
+    const float dx = fmaxf(0.f, fmaxf(r.x - c.z, c.x - r.z));
+    const float dy = fmaxf(0.f, fmaxf(r.y - c.w, c.y - r.w));
+    return fmaf(dx, dx, dy * dy) > tau2;
+}
 
 // rho of token i of one sample from the partial sums of the tiles that hold it, in a fixed order (reproducible
 // bits): the row-side slots of the column tiles that pair row tile i / 128 with later tokens, then the column-side
