@@ -437,7 +437,10 @@ def test_filter_resident_shapes(B, n, metric, check):
 # Long samples (8192 tokens and more) keep the Gram tiles of the density sweep and run Eq. 3 as a separate pass over
 # them: a ragged length (tiles that straddle the diagonal and the end of the sample), both metrics, with and
 # without the spatial test.  Small feature width: the oracle's pairwise work stays cheap.
-@pytest.mark.parametrize("n,metric,tau", [(8200, 0, 0.6), (8321, 1, 0.6), (8200, 0, -1.0), (8192, 0, 0.25)])
+# With a radius, the tiles whose row block lies beyond it from their column blocks are neither kept nor read: 0.25 and
+# 0.02 drop most of them (0.02: nearly all but the tiles on the diagonal).
+@pytest.mark.parametrize("n,metric,tau", [(8200, 0, 0.6), (8321, 1, 0.6), (8200, 0, -1.0), (8192, 0, 0.25),
+                                          (8250, 0, 0.02), (8200, 1, 0.25)])
 def test_filter_long_sample_delta_pass(n, metric, tau):
     w = dataclasses.replace(W.workload("c4"), B=1, D=64, dup_rate=0.3)
     f = W.make_features(w, n=n, B=1)
@@ -449,6 +452,22 @@ def test_filter_long_sample_delta_pass(n, metric, tau):
     rep = []
     check_vic_sample(f[0], p[0], metric, d_c, tau, nc, g.rho[0], g.delta2[0], g.parent[0], g.label[0], rep)
     print("filter long sample", n, metric, tau, rep)
+
+
+def test_filter_long_samples_scattered_positions():
+    """Two long samples in one call, one with positions in no order at all (no tile lies beyond the radius), one on the
+    grid with a token whose position is not a number (it can be nobody's neighbour)."""
+    n = 8192
+    w = dataclasses.replace(W.workload("c4"), B=2, D=64, dup_rate=0.3)
+    f = W.make_features(w, n=n, B=2)
+    p = W.make_positions(w, n)[:2].copy()
+    p[0] = np.random.default_rng(5).random((n, 2), dtype=np.float32)
+    p[1, 4000] = np.nan
+    nc = n // 20
+    g = gpu_filter(f, p, 0, w.d_c, 0.3, nc)
+    assert g.status == vb.OK and np.all(g.n_clusters == nc)
+    for b in range(2):
+        check_vic_sample(f[b], p[b], 0, w.d_c, 0.3, nc, g.rho[b], g.delta2[b], g.parent[b], g.label[b])
 
 
 def test_filter_edge_cases():
