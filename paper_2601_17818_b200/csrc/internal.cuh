@@ -134,6 +134,23 @@ __device__ __forceinline__ uint32_t block_exclusive_sum(uint32_t v, uint32_t* wa
     return base + incl - v;
 }
 
+// Exclusive prefix of one value per warp (uniform inside the warp) over the 32 warps of a CTA of 1024 threads; `total` = the sum.
+__device__ __forceinline__ uint32_t warp_totals_scan(uint32_t warp_total, uint32_t* warp_sums, uint32_t& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) warp_sums[warp] = warp_total;
+    __syncthreads();
+    uint32_t v = warp_sums[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += t;
+    }
+    total = __shfl_sync(0xffffffffu, v, 31);
+    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
+    __syncthreads();
+    return warp == 0 ? 0u : base;
+}
+
 #endif
 
 }  // namespace vitcop

@@ -35,23 +35,6 @@ constexpr int kCntEntries = kPlanWarps * kCntStride;
 // rolled loops on purpose: the kernel runs once per call on a handful of SMs, so every instruction it executes is
 // fetched cold, and a loop body fetched once beats sixteen unrolled copies.
 
-// Exclusive prefix of one value per warp (uniform inside the warp) over the CTA's 32 warps; `total` = the sum.
-__device__ __forceinline__ uint32_t warp_totals_scan(uint32_t warp_total, uint32_t* warp_sums, uint32_t& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) warp_sums[warp] = warp_total;
-    __syncthreads();
-    uint32_t v = warp_sums[lane];
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
-    }
-    total = __shfl_sync(0xffffffffu, v, 31);
-    const uint32_t base = __shfl_sync(0xffffffffu, v, (warp + 31) & 31);
-    __syncthreads();
-    return warp == 0 ? 0u : base;
-}
-
 // One walk of a warp over its items with a cursor per (digit, warp) in `cnt`: every item receives the cursor of its
 // digit plus the number of items of the same digit in front of it in its row, and the cursor moves past the row's
 // items.  With the cursors at zero the walk counts (dst null); with the cursors at their scanned values it writes the

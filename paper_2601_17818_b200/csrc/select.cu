@@ -21,7 +21,7 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     uint32_t* keys = smem_u32;
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_sums[kSelWarps];
-    __shared__ uint32_t s_digit, s_krem, s_whole;
+    __shared__ uint32_t s_digit, s_krem, s_whole, s_lo, s_hi;
 
     // The compaction that follows may start at once: it copies the rows that do not depend on the selection and
     // waits for this kernel to complete before it reads the kept indices.
@@ -36,17 +36,37 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     keep_idx += (int64_t)b * keep_stride;
     if (keep_mask) keep_mask += (int64_t)b * Nv_cap;
 
-    for (int i = tid; i < n; i += kSelThreads) keys[i] = order_key(score[i], largest);
+    if (tid == 0) { s_lo = 0xFFFFFFFFu; s_hi = 0u; }
+    __syncthreads();
+    {
+        uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+        for (int i = tid; i < n; i += kSelThreads) {
+            const uint32_t key = order_key(score[i], largest);
+            keys[i] = key;
+            lo = min(lo, key);
+            hi = max(hi, key);
+        }
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        if (lane == 0 && lo <= hi) {
+            atomicMin(&s_lo, lo);
+            atomicMax(&s_hi, hi);
+        }
+    }
     __syncthreads();
 
     uint32_t T = 0xFFFFFFFFu;   // cut key: keep key < T, plus `krem` of the key == T elements
     uint32_t krem = 0;
     if (k > 0 && k < n) {
-        uint32_t prefix = 0;
+        // The keys of a sample share their leading bits (norms of one layer lie within a few octaves): the passes
+        // start at the highest bit in which two keys differ, eight bits at a time down to bit 0.
+        const int top = 32 - __clz(s_lo ^ s_hi);            // bits [top, 32) are common to all keys; 0: all keys equal
+        uint32_t prefix = top >= 32 ? 0u : (s_hi >> top) << top;
         krem = (uint32_t)k;
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            const uint32_t hi_mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        for (int hi_bit = top; hi_bit > 0; hi_bit -= 8) {
+            const int shift = hi_bit > 8 ? hi_bit - 8 : 0;
+            const uint32_t digit_mask = (1u << (hi_bit - shift)) - 1u;
+            const uint32_t hi_mask = hi_bit >= 32 ? 0u : (0xFFFFFFFFu << hi_bit);
             if (tid < 256) hist[tid] = 0;
             __syncthreads();
             for (int base = 0; base < n; base += kSelThreads) {
@@ -54,7 +74,7 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
                 int dig = -1;
                 if (i < n) {
                     const uint32_t key = keys[i];
-                    if ((key & hi_mask) == prefix) dig = (int)((key >> shift) & 255u);
+                    if ((key & hi_mask) == prefix) dig = (int)((key >> shift) & digit_mask);
                 }
                 const uint32_t peers = __match_any_sync(0xffffffffu, dig);
                 if (dig >= 0 && lane == __ffs(peers) - 1) atomicAdd(&hist[dig], (uint32_t)__popc(peers));
@@ -101,22 +121,40 @@ select_plain_kernel(const float* __restrict__ score, const int32_t* __restrict__
     } else if (k >= n) {
         kept = emit_ascending(n, [](int) { return true; }, keep_idx, keep_stride, keep_mask, warp_sums);
     } else {
-        // one sweep in index order: rank among the elements equal to the cut, then rank among the kept
-        uint32_t eq_running = 0, keep_running = 0;
-        for (int base = 0; base < n; base += kSelThreads) {
-            const int i = base + tid;
+        // Ranks in index order -- first among the elements equal to the cut, then among the kept -- with two scans for
+        // the whole sample: warp w owns the tokens [w * 32 E, (w + 1) * 32 E) and takes them 32 at a time, so that a
+        // ballot gives the rank inside a row and one scan over the 32 warp totals the rest.
+        const int E = (n + kSelThreads - 1) / kSelThreads;
+        const uint32_t lt = (1u << lane) - 1u;
+        uint32_t weq = 0;
+        for (int e = 0; e < E; ++e) {
+            const int i = (warp * E + e) * 32 + lane;
+            weq += __popc(__ballot_sync(0xffffffffu, i < n && keys[i] == T));
+        }
+        uint32_t total;
+        uint32_t eq_run = warp_totals_scan(weq, warp_sums, total);
+        uint32_t fbits = 0, wkeep = 0;                     // bit e: this thread's token of row e is kept
+        for (int e = 0; e < E; ++e) {
+            const int i = (warp * E + e) * 32 + lane;
             const uint32_t key = i < n ? keys[i] : 0xFFFFFFFFu;
             const bool eq = i < n && key == T;
-            uint32_t eq_total, keep_total;
-            const uint32_t eq_rank = eq_running + block_prefix_count(eq, warp_sums, eq_total);
-            const bool f = i < n && (key < T || (eq && eq_rank < krem));
-            const uint32_t r = keep_running + block_prefix_count(f, warp_sums, keep_total);
-            if (f && r < (uint32_t)keep_stride) keep_idx[r] = i;
-            if (keep_mask && i < n) keep_mask[i] = f ? 1 : 0;
-            eq_running += eq_total;
-            keep_running += keep_total;
+            const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+            const bool f = i < n && (key < T || (eq && eq_run + __popc(bal & lt) < krem));
+            eq_run += __popc(bal);
+            fbits |= (uint32_t)f << e;
+            wkeep += __popc(__ballot_sync(0xffffffffu, f));
         }
-        kept = keep_running;
+        uint32_t r = warp_totals_scan(wkeep, warp_sums, total);
+        for (int e = 0; e < E; ++e) {
+            const int i = (warp * E + e) * 32 + lane;
+            const bool f = (fbits >> e & 1u) != 0;
+            const uint32_t bal = __ballot_sync(0xffffffffu, f);
+            const uint32_t at = r + __popc(bal & lt);
+            if (f && at < (uint32_t)keep_stride) keep_idx[at] = i;
+            if (keep_mask && i < n) keep_mask[i] = f ? 1 : 0;
+            r += __popc(bal);
+        }
+        kept = total;
     }
     if (tid == 0) n_keep[b] = (int32_t)kept;
 }
